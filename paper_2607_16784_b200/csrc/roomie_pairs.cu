@@ -1,0 +1,663 @@
+// Pairwise interference (Algorithm 1, lines 6-20): plan -> tile walk -> finalize.
+//
+// The event-driven walk over two kernel timelines is a merge of the two sorted lists of kernel
+// end times: every walk iteration consumes the kernel that ends first.  That makes the walk a
+// merge path, which can be cut at any diagonal by a binary search, so one walk is split into
+// tiles of kTileItems path steps and each tile into per-thread slices.  The delay sums are
+// order-free (every overlapping pairing is met exactly once), so tiles are summed afterwards
+// in a fixed order and the result does not depend on how the path was cut.
+//
+//   plan      one thread per (pair, alignment): alignment kept?  path length, tiles, and the
+//             path split point of every tile (binary searches on the global records)
+//   tiles     one CTA per tile: stage the tile's records in shared memory, per-thread merge
+//             path search + kItems sequential steps, warp-shuffle reduction -> one partial
+//   finalize  one CTA per pair: sum partials per alignment, median over alignments, gamma, /T
+#include "roomie_common.cuh"
+
+namespace roomie {
+
+constexpr int kTileThreads = 128;
+constexpr int kItems = 16;                              // path steps per thread
+constexpr int kTileItems = kTileThreads * kItems;       // path steps per tile
+constexpr int kFinalThreads = 128;
+
+struct PairSet {                  // which pairs a launch covers
+    uint64_t pair_begin;          // first triangular pair index (explicit == 0)
+    uint32_t n_pairs;
+    uint32_t explicit_pair;       // 1: the single ordered pair (a, b)
+    uint32_t a, b;
+};
+
+struct LibView {
+    const uint4* records;
+    const uint32_t* offsets;
+    const unsigned long long* T;
+    uint32_t P;
+    PhiCap cap;
+};
+
+__device__ __forceinline__ void pair_of(const PairSet& ps, uint32_t P, uint32_t local, uint32_t& a, uint32_t& b) {
+    if (ps.explicit_pair) { a = ps.a; b = ps.b; return; }
+    const unsigned long long p = ps.pair_begin + local;
+    // row a of the upper triangle starts at a*P - a(a-1)/2
+    const double n = 2.0 * P + 1.0;
+    long long r = (long long)((n - sqrt(n * n - 8.0 * (double)p)) * 0.5);
+    if (r < 0) r = 0;
+    if (r > (long long)P - 1) r = P - 1;
+    auto row_start = [P](long long x) { return (unsigned long long)(x * P - x * (x - 1) / 2); };
+    while (r > 0 && row_start(r) > p) --r;
+    while (r + 1 < (long long)P && row_start(r + 1) <= p) ++r;
+    a = (uint32_t)r;
+    b = a + (uint32_t)(p - row_start(r));
+}
+
+// alignment grid of one model: |G(q, A)| and its c-th element (A = 0: every index)
+__device__ __forceinline__ uint32_t grid_count(uint32_t q, uint32_t A) { return (A == 0 || A > q) ? q : A; }
+__device__ __forceinline__ uint32_t grid_start(uint32_t q, uint32_t A, uint32_t c) {
+    return (A == 0 || A > q) ? c : (uint32_t)(((unsigned long long)c * q) / A);
+}
+
+struct PlanArgs {
+    LibView lib;
+    PairSet ps;
+    uint32_t slots;          // alignment slots per pair
+    uint32_t n_align;
+    int start_filter;
+    int lockstep;
+    WalkInfo* walks;
+    TileDesc* tiles;
+    uint32_t* tile_counter;  // [0] tiles allocated so far
+    uint32_t tile_capacity;
+    uint32_t* status;
+};
+
+// merge-path split: number of A records among the first d merged items; A goes first on equal
+// end times.  Keys are end ticks re-based to the alignment's start.
+__device__ __forceinline__ uint32_t path_split_global(const uint4* __restrict__ A, const uint4* __restrict__ B,
+                                                      uint32_t na, uint32_t nb, uint32_t baseA, uint32_t baseB,
+                                                      uint32_t d) {
+    uint32_t lo = d > nb ? d - nb : 0u, hi = d < na ? d : na;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        const uint32_t ea = __ldg(&A[mid].y) - baseA;
+        const uint32_t eb = __ldg(&B[d - 1 - mid].y) - baseB;
+        if (ea <= eb) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(256) plan_kernel(PlanArgs g) {
+    const unsigned long long w = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned long long n_walks = (unsigned long long)g.ps.n_pairs * g.slots;
+    const int lane = threadIdx.x & 31;
+    bool valid = w < n_walks;
+    uint32_t a = 0, b = 0, offa = 0, offb = 0, si = 0, sj = 0, na = 0, nb = 0, baseA = 0, baseB = 0;
+    uint32_t L = 0, n_tiles = 0;
+    const uint4 *RA = nullptr, *RB = nullptr;
+    if (valid) {
+        const uint32_t local = (uint32_t)(w / g.slots), c = (uint32_t)(w % g.slots);
+        pair_of(g.ps, g.lib.P, local, a, b);
+        offa = g.lib.offsets[a]; offb = g.lib.offsets[b];
+        const uint32_t qa = g.lib.offsets[a + 1] - offa, qb = g.lib.offsets[b + 1] - offb;
+        const uint32_t ga = grid_count(qa, g.n_align), gb = grid_count(qb, g.n_align);
+        const uint32_t ca = c / gb, cb = c % gb;
+        valid = ca < ga;
+        if (valid) {
+            si = grid_start(qa, g.n_align, ca);
+            sj = grid_start(qb, g.n_align, cb);
+            RA = g.lib.records + offa + si;
+            RB = g.lib.records + offb + sj;
+            const uint4 ra = __ldg(RA), rb = __ldg(RB);
+            if (g.start_filter)
+                valid = phi_exceeds(g.lib.cap.lo - ra.z, g.lib.cap.hi - ra.w, rb.z, rb.w);
+            na = qa - si; nb = qb - sj;
+            baseA = ra.x; baseB = rb.x;
+        }
+        if (valid) {
+            if (g.lockstep) {
+                L = na < nb ? na : nb;
+            } else {
+                // the walk ends when one model runs out: count the path states up to there
+                const uint32_t endA = __ldg(&RA[na - 1].y) - baseA, endB = __ldg(&RB[nb - 1].y) - baseB;
+                if (endA <= endB) {          // A runs out first: B kernels ending strictly before
+                    uint32_t lo = 0, hi = nb;
+                    while (lo < hi) {
+                        const uint32_t mid = (lo + hi) >> 1;
+                        if (__ldg(&RB[mid].y) - baseB < endA) lo = mid + 1; else hi = mid;
+                    }
+                    L = na + lo;
+                } else {                     // B runs out first: A kernels ending at or before
+                    uint32_t lo = 0, hi = na;
+                    while (lo < hi) {
+                        const uint32_t mid = (lo + hi) >> 1;
+                        if (__ldg(&RA[mid].y) - baseA <= endB) lo = mid + 1; else hi = mid;
+                    }
+                    L = nb + lo;
+                }
+            }
+            n_tiles = (L + kTileItems - 1) / kTileItems;
+        }
+    }
+    // warp-aggregated allocation of tile slots
+    uint32_t incl = n_tiles;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, s);
+        if (lane >= s) incl += up;
+    }
+    const uint32_t warp_total = __shfl_sync(0xffffffffu, incl, 31);
+    uint32_t base = 0;
+    if (lane == 31 && warp_total) base = atomicAdd(g.tile_counter, warp_total);
+    base = __shfl_sync(0xffffffffu, base, 31) + incl - n_tiles;
+    if (w < n_walks) {
+        WalkInfo wi;
+        wi.tile_base = base; wi.n_tiles = n_tiles; wi.length = L; wi.valid = valid ? 1u : 0u;
+        g.walks[w] = wi;
+    }
+    if (!valid || n_tiles == 0) return;
+    if (base + n_tiles > g.tile_capacity) {          // never expected: the host sizes the list
+        atomicOr(g.status, ROOMIE_FLAG_WORKSPACE);
+        g.walks[w].n_tiles = 0;
+        TileDesc z;
+        z.recA = z.recB = z.cntA = z.cntB = z.baseA = z.baseB = z.flags = 0; z.walk = (uint32_t)w;
+        for (uint32_t k = 0; k < n_tiles && base + k < g.tile_capacity; ++k) g.tiles[base + k] = z;
+        return;
+    }
+    uint32_t x0 = 0;
+    for (uint32_t k = 0; k < n_tiles; ++k) {
+        const uint32_t d0 = k * kTileItems;
+        const uint32_t d1 = (d0 + kTileItems < L) ? d0 + kTileItems : L;
+        uint32_t x1;
+        if (g.lockstep) x1 = d1;
+        else if (d1 == L) {
+            // end of the walk: whichever side ran out
+            const uint32_t endA = __ldg(&RA[na - 1].y) - baseA, endB = __ldg(&RB[nb - 1].y) - baseB;
+            x1 = (endA <= endB) ? na : L - nb;
+        } else x1 = path_split_global(RA, RB, na, nb, baseA, baseB, d1);
+        TileDesc t;
+        if (g.lockstep) {
+            t.recA = offa + si + d0; t.recB = offb + sj + d0;
+            t.cntA = d1 - d0; t.cntB = d1 - d0;
+            t.flags = 0;
+        } else {
+            const uint32_t y0 = d0 - x0, y1 = d1 - x1;
+            t.recA = offa + si + x0; t.recB = offb + sj + y0;
+            t.cntA = x1 - x0; t.cntB = y1 - y0;
+            t.flags = (x1 < na ? 1u : 0u) | (y1 < nb ? 2u : 0u);
+        }
+        t.baseA = baseA; t.baseB = baseB;
+        t.walk = (uint32_t)w;
+        g.tiles[base + k] = t;
+        x0 = x1;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// TIMELINE tiles
+// ---------------------------------------------------------------------------------------
+struct TileArgs {
+    const uint4* records;
+    const TileDesc* tiles;
+    const uint32_t* tile_counter;
+    uint32_t tile_capacity;
+    TilePartial* partials;
+    const float2* share_table;
+    uint32_t Wt;                 // W + 1
+    PhiCap cap;
+};
+
+__device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned long long V, uint32_t ties,
+                                                   TilePartial* out, float* s_f, unsigned long long* s_v,
+                                                   uint32_t* s_t, int nwarps) {
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        di += __shfl_xor_sync(0xffffffffu, di, s);
+        dj += __shfl_xor_sync(0xffffffffu, dj, s);
+        V += __shfl_xor_sync(0xffffffffu, V, s);
+        ties += __shfl_xor_sync(0xffffffffu, ties, s);
+    }
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) { s_f[2 * wid] = di; s_f[2 * wid + 1] = dj; s_v[wid] = V; s_t[wid] = ties; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        TilePartial p;
+        p.di = 0.0f; p.dj = 0.0f; p.V = 0; p.ties = 0; p.pad = 0;
+        for (int w = 0; w < nwarps; ++w) { p.di += s_f[2 * w]; p.dj += s_f[2 * w + 1]; p.V += s_v[w]; p.ties += s_t[w]; }
+        *out = p;
+    }
+}
+
+__global__ void __launch_bounds__(kTileThreads) timeline_tiles_kernel(TileArgs g) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2* s_tab = reinterpret_cast<float2*>(smem_raw);
+    uint4* s_rec = reinterpret_cast<uint4*>(smem_raw + (((size_t)g.Wt * g.Wt * sizeof(float2) + 15) & ~(size_t)15));
+    __shared__ float s_f[2 * kTileThreads / 32];
+    __shared__ unsigned long long s_v[kTileThreads / 32];
+    __shared__ uint32_t s_t[kTileThreads / 32];
+
+    for (uint32_t i = threadIdx.x; i < g.Wt * g.Wt; i += kTileThreads) s_tab[i] = __ldg(&g.share_table[i]);
+    const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
+
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const TileDesc d = g.tiles[t];
+        const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
+        __syncthreads();                                   // previous tile fully consumed
+        for (uint32_t i = threadIdx.x; i < loadA + loadB; i += kTileThreads)
+            s_rec[i] = __ldg(i < loadA ? &g.records[d.recA + i] : &g.records[d.recB + (i - loadA)]);
+        __syncthreads();
+        const uint4* sA = s_rec;
+        const uint4* sB = s_rec + loadA;
+        const uint32_t len = d.cntA + d.cntB;
+        const uint32_t diag = threadIdx.x * kItems;
+        float di = 0.0f, dj = 0.0f;
+        unsigned long long V = 0;
+        uint32_t ties = 0;
+        if (diag < len) {
+            // this thread's start point on the tile's merge path
+            uint32_t lo = diag > d.cntB ? diag - d.cntB : 0u, hi = diag < d.cntA ? diag : d.cntA;
+            while (lo < hi) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (sA[mid].y - d.baseA <= sB[diag - 1 - mid].y - d.baseB) lo = mid + 1; else hi = mid;
+            }
+            uint32_t x = lo, y = diag - lo;
+            const uint32_t steps = (len - diag < (uint32_t)kItems) ? len - diag : (uint32_t)kItems;
+            const uint32_t tie_limit = d.cntA + (d.flags & 1u);     // x + 1 < tie_limit: A has a next kernel
+            uint4 ra = sA[x], rb = sB[y];
+            int32_t Sa = (int32_t)(ra.x - d.baseA), Ea = (int32_t)(ra.y - d.baseA);
+            int32_t Sb = (int32_t)(rb.x - d.baseB), Eb = (int32_t)(rb.y - d.baseB);
+#pragma unroll
+            for (int s = 0; s < kItems; ++s) {
+                if ((uint32_t)s < steps) {
+                    const int32_t ov = min(Ea, Eb) - max(Sa, Sb);
+                    const bool hit = (ov > 0) && phi_exceeds(g.cap.lo - ra.z, g.cap.hi - ra.w, rb.z, rb.w);
+                    const float2 w = s_tab[(ra.z >> kWarpShift) * g.Wt + (rb.z >> kWarpShift)];
+                    const float ovf = hit ? (float)ov : 0.0f;
+                    di = fmaf(ovf, w.x, di);
+                    dj = fmaf(ovf, w.y, dj);
+                    V += hit ? (unsigned long long)(uint32_t)ov : 0ull;
+                    const bool adv_a = Ea <= Eb;
+                    ties += (Ea == Eb && x + 1 < tie_limit) ? 1u : 0u;
+                    if (adv_a) {
+                        ++x; ra = sA[x];
+                        Sa = (int32_t)(ra.x - d.baseA); Ea = (int32_t)(ra.y - d.baseA);
+                    } else {
+                        ++y; rb = sB[y];
+                        Sb = (int32_t)(rb.x - d.baseB); Eb = (int32_t)(rb.y - d.baseB);
+                    }
+                }
+            }
+        }
+        block_reduce_store(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// LOCKSTEP tiles (Algorithm 1 as printed): pairing t of the walk is (s_i + t, s_j + t)
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kTileThreads) lockstep_tiles_kernel(TileArgs g) {
+    __shared__ float s_f[2 * kTileThreads / 32];
+    __shared__ unsigned long long s_v[kTileThreads / 32];
+    __shared__ uint32_t s_t[kTileThreads / 32];
+    const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const TileDesc d = g.tiles[t];
+        float di = 0.0f, dj = 0.0f;
+        unsigned long long V = 0;
+        for (uint32_t i = threadIdx.x; i < d.cntA; i += kTileThreads) {
+            const uint4 ra = __ldg(&g.records[d.recA + i]), rb = __ldg(&g.records[d.recB + i]);
+            if (phi_exceeds(g.cap.lo - ra.z, g.cap.hi - ra.w, rb.z, rb.w)) {
+                const float2 w = __ldg(&g.share_table[(ra.z >> kWarpShift) * g.Wt + (rb.z >> kWarpShift)]);
+                const uint32_t da = ra.y - ra.x, db = rb.y - rb.x;
+                di = fmaf((float)da, w.x, di);
+                dj = fmaf((float)db, w.y, dj);
+                V += (unsigned long long)da + db;
+            }
+        }
+        __syncthreads();
+        block_reduce_store(di, dj, V, 0u, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// finalize: one CTA per pair
+// ---------------------------------------------------------------------------------------
+struct FinalArgs {
+    LibView lib;
+    PairSet ps;
+    uint32_t slots;
+    uint32_t n_align;
+    const WalkInfo* walks;
+    const TilePartial* partials;
+    float* P_out;                 // matrix [P*P] (or out2 for an explicit pair)
+    unsigned long long* evals_out;
+    roomie_pair_detail detail;    // capacity 0 = none
+};
+
+// k-th smallest of v[0..n) by rank counting (ties ordered by index); every thread returns it
+__device__ float select_rank(const float* v, uint32_t n, uint32_t k, float* s_pick) {
+    for (uint32_t e = threadIdx.x; e < n; e += kFinalThreads) {
+        const float x = v[e];
+        uint32_t rank = 0;
+        for (uint32_t j = 0; j < n; ++j) {
+            const float y = v[j];
+            rank += (y < x) || (y == x && j < e);
+        }
+        if (rank == k) *s_pick = x;
+    }
+    __syncthreads();
+    const float r = *s_pick;
+    __syncthreads();
+    return r;
+}
+
+__global__ void __launch_bounds__(kFinalThreads) finalize_kernel(FinalArgs g) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* v_i = reinterpret_cast<float*>(smem_raw);
+    float* v_j = v_i + g.slots;
+    __shared__ uint32_t s_warp[kFinalThreads / 32];
+    __shared__ float s_pick;
+    __shared__ unsigned long long s_ev[kFinalThreads / 32];
+
+    const uint32_t local = blockIdx.x;
+    uint32_t a, b;
+    pair_of(g.ps, g.lib.P, local, a, b);
+    const uint32_t qa = g.lib.offsets[a + 1] - g.lib.offsets[a], qb = g.lib.offsets[b + 1] - g.lib.offsets[b];
+    const uint32_t gb = grid_count(qb, g.n_align);
+    const WalkInfo* walks = g.walks + (size_t)local * g.slots;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+
+    uint32_t kept_before = 0;
+    unsigned long long evals = 0;
+    for (uint32_t c0 = 0; c0 < g.slots; c0 += kFinalThreads) {
+        const uint32_t c = c0 + threadIdx.x;
+        bool valid = false;
+        float di = 0.0f, dj = 0.0f;
+        unsigned long long V = 0;
+        uint32_t ev = 0;
+        if (c < g.slots) {
+            const WalkInfo wi = walks[c];
+            valid = wi.valid != 0;
+            if (valid) {
+                uint32_t ties = 0;
+                for (uint32_t k = 0; k < wi.n_tiles; ++k) {          // fixed order: tile 0, 1, ...
+                    const TilePartial p = g.partials[wi.tile_base + k];
+                    di += p.di; dj += p.dj; V += p.V; ties += p.ties;
+                }
+                ev = wi.length - ties;
+                evals += ev;
+            }
+        }
+        // ordered compaction of the kept alignments
+        const uint32_t ballot = __ballot_sync(0xffffffffu, valid);
+        if (lane == 0) s_warp[wid] = __popc(ballot);
+        __syncthreads();
+        uint32_t pos = kept_before + __popc(ballot & ((1u << lane) - 1u));
+        uint32_t chunk = 0;
+#pragma unroll
+        for (int w = 0; w < kFinalThreads / 32; ++w) { if (w < wid) pos += s_warp[w]; chunk += s_warp[w]; }
+        if (valid) {
+            v_i[pos] = di; v_j[pos] = dj;
+            if (pos < g.detail.capacity) {
+                const uint32_t ca = c / gb, cb = c % gb;
+                if (g.detail.s_i) g.detail.s_i[pos] = grid_start(qa, g.n_align, ca);
+                if (g.detail.s_j) g.detail.s_j[pos] = grid_start(qb, g.n_align, cb);
+                if (g.detail.delta_i) g.detail.delta_i[pos] = di;
+                if (g.detail.delta_j) g.detail.delta_j[pos] = dj;
+                if (g.detail.V) g.detail.V[pos] = V;
+                if (g.detail.evals) g.detail.evals[pos] = ev;
+            }
+        }
+        kept_before += chunk;
+        __syncthreads();
+    }
+    const uint32_t n = kept_before;
+    float med_i = 0.0f, med_j = 0.0f;
+    if (n > 0) {
+        const uint32_t k1 = (n - 1) / 2, k2 = n / 2;
+        const float i1 = select_rank(v_i, n, k1, &s_pick);
+        const float i2 = (k2 == k1) ? i1 : select_rank(v_i, n, k2, &s_pick);
+        const float j1 = select_rank(v_j, n, k1, &s_pick);
+        const float j2 = (k2 == k1) ? j1 : select_rank(v_j, n, k2, &s_pick);
+        med_i = 0.5f * (i1 + i2);
+        med_j = 0.5f * (j1 + j2);
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) evals += __shfl_xor_sync(0xffffffffu, evals, s);
+    if (lane == 0) s_ev[wid] = evals;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned long long Ta = g.lib.T[a], Tb = g.lib.T[b];
+        const float fa = (float)qa, fb = (float)qb;
+        const float g_ab = fmaxf(__fdiv_rn(fa, fb), 1.0f), g_ba = fmaxf(__fdiv_rn(fb, fa), 1.0f);
+        const float p_ab = Ta ? __fdiv_rn(g_ab * med_i, (float)Ta) : 0.0f;
+        const float p_ba = Tb ? __fdiv_rn(g_ba * med_j, (float)Tb) : 0.0f;
+        if (g.ps.explicit_pair) {
+            g.P_out[0] = p_ab; g.P_out[1] = p_ba;
+        } else {
+            g.P_out[(size_t)a * g.lib.P + b] = p_ab;
+            if (a != b) g.P_out[(size_t)b * g.lib.P + a] = p_ba;
+        }
+        if (g.detail.n_kept) *g.detail.n_kept = n;
+        if (g.evals_out) {
+            unsigned long long tot = 0;
+            for (int w = 0; w < kFinalThreads / 32; ++w) tot += s_ev[w];
+            atomicAdd(g.evals_out, tot);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+struct PairRange { uint32_t a, b; };
+
+static void pair_of_host(uint64_t p, uint32_t P, uint32_t& a, uint32_t& b) {
+    uint64_t r = 0, start = 0;
+    // rows shrink by one each; walk rows (P is at most a few thousand, and this runs once per batch edge)
+    while (r + 1 < P && start + (P - r) <= p) { start += P - r; ++r; }
+    a = (uint32_t)r; b = (uint32_t)(r + (p - start));
+}
+
+static uint32_t host_grid_count(uint32_t q, uint32_t A) { return (A == 0 || A > q) ? q : A; }
+
+struct Need { uint64_t walks, tiles; };
+
+// upper bound of walk slots and tiles for pairs [p0, p1): a walk of a pair has at most
+// q_a + q_b - 1 steps whatever its alignment
+static bool batch_need(const roomie_library* lib, const roomie_opts* o, bool explicit_pair, uint32_t ea, uint32_t eb,
+                       uint64_t p0, uint64_t p1, uint32_t slots, Need& need) {
+    const uint32_t* off = lib->offsets_host;
+    uint64_t tiles = 0;
+    auto add = [&](uint32_t a, uint32_t b) {
+        const uint32_t qa = off[a + 1] - off[a], qb = off[b + 1] - off[b];
+        const uint64_t n = (uint64_t)host_grid_count(qa, o->n_align) * host_grid_count(qb, o->n_align);
+        const uint64_t per = o->walk_mode == ROOMIE_WALK_LOCKSTEP
+                                 ? ((uint64_t)(qa < qb ? qa : qb) + kTileItems - 1) / kTileItems
+                                 : ((uint64_t)qa + qb - 1 + kTileItems - 1) / kTileItems;
+        tiles += n * per;
+    };
+    if (explicit_pair) add(ea, eb);
+    else {
+        uint32_t a, b;
+        pair_of_host(p0, lib->num_profiles, a, b);
+        for (uint64_t p = p0; p < p1; ++p) {
+            add(a, b);
+            if (++b == lib->num_profiles) { ++a; b = a; }
+        }
+    }
+    need.walks = (explicit_pair ? 1 : (p1 - p0)) * (uint64_t)slots;
+    need.tiles = tiles;
+    return true;
+}
+
+static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static size_t bytes_for(const Need& n) {
+    return 256 + align_up(n.walks * sizeof(WalkInfo)) + align_up(n.tiles * sizeof(TileDesc)) +
+           align_up(n.tiles * sizeof(TilePartial));
+}
+
+static int slots_for(const roomie_library* lib, const roomie_opts* o, bool explicit_pair, uint32_t ea, uint32_t eb,
+                     uint32_t& slots) {
+    if (o->n_align > 0) {
+        if ((uint64_t)o->n_align * o->n_align > kMaxAlignSlots) return ROOMIE_ERR_CAPACITY;
+        slots = o->n_align * o->n_align;
+        return ROOMIE_OK;
+    }
+    // full Cartesian product: the largest q_a * q_b among the pairs involved
+    const uint32_t* off = lib->offsets_host;
+    uint64_t m;
+    if (explicit_pair) m = (uint64_t)(off[ea + 1] - off[ea]) * (off[eb + 1] - off[eb]);
+    else {
+        uint64_t q1 = 0;
+        for (uint32_t p = 0; p < lib->num_profiles; ++p) { const uint64_t q = off[p + 1] - off[p]; if (q > q1) q1 = q; }
+        m = q1 * q1;
+    }
+    if (m > kMaxAlignSlots) return ROOMIE_ERR_CAPACITY;
+    slots = (uint32_t)m;
+    return ROOMIE_OK;
+}
+
+static int check_lib(const roomie_library* lib, const roomie_opts* o) {
+    if (!lib || !o || !lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->share_table ||
+        !lib->status || lib->num_profiles == 0)
+        return ROOMIE_ERR_INVALID_ARG;
+    if (o->walk_mode != ROOMIE_WALK_TIMELINE && o->walk_mode != ROOMIE_WALK_LOCKSTEP) return ROOMIE_ERR_INVALID_ARG;
+    return validate_spec(&lib->spec);
+}
+
+static int run_batch(const roomie_library* lib, const roomie_opts* o, const PairSet& ps, uint32_t slots,
+                     const Need& need, float* P_out, uint64_t* evals_out, const roomie_pair_detail* detail,
+                     unsigned char* ws, cudaStream_t st) {
+    uint32_t* counter = reinterpret_cast<uint32_t*>(ws);
+    WalkInfo* walks = reinterpret_cast<WalkInfo*>(ws + 256);
+    TileDesc* tiles = reinterpret_cast<TileDesc*>(ws + 256 + align_up(need.walks * sizeof(WalkInfo)));
+    TilePartial* partials = reinterpret_cast<TilePartial*>(reinterpret_cast<unsigned char*>(tiles) +
+                                                           align_up(need.tiles * sizeof(TileDesc)));
+    ROOMIE_CUDA_OK(cudaMemsetAsync(counter, 0, 256, st));
+    LibView lv;
+    lv.records = static_cast<const uint4*>(lib->records);
+    lv.offsets = lib->offsets;
+    lv.T = reinterpret_cast<const unsigned long long*>(lib->T);
+    lv.P = lib->num_profiles;
+    lv.cap = make_cap(lib->spec);
+
+    PlanArgs pa;
+    pa.lib = lv; pa.ps = ps; pa.slots = slots; pa.n_align = o->n_align; pa.start_filter = o->start_filter;
+    pa.lockstep = o->walk_mode == ROOMIE_WALK_LOCKSTEP;
+    pa.walks = walks; pa.tiles = tiles; pa.tile_counter = counter;
+    pa.tile_capacity = (uint32_t)need.tiles; pa.status = lib->status;
+    const uint64_t plan_blocks = (need.walks + 255) / 256;
+    plan_kernel<<<(unsigned)plan_blocks, 256, 0, st>>>(pa);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+
+    TileArgs ta;
+    ta.records = lv.records; ta.tiles = tiles; ta.tile_counter = counter; ta.tile_capacity = (uint32_t)need.tiles; ta.partials = partials;
+    ta.share_table = reinterpret_cast<const float2*>(lib->share_table);
+    ta.Wt = lib->spec.threads_per_sm / 32u + 1u; ta.cap = lv.cap;
+    profile_mark(st, true);
+    if (pa.lockstep) {
+        uint64_t grid = (uint64_t)sm_count() * 8;
+        if (grid > need.tiles) grid = need.tiles ? need.tiles : 1;
+        lockstep_tiles_kernel<<<(unsigned)grid, kTileThreads, 0, st>>>(ta);
+    } else {
+        const size_t tab = ((size_t)ta.Wt * ta.Wt * sizeof(float2) + 15) & ~(size_t)15;
+        const size_t smem = tab + (size_t)(kTileItems + 4) * sizeof(uint4);
+        if (smem > 227 * 1024) return ROOMIE_ERR_CAPACITY;
+        if (smem > 48 * 1024)
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(timeline_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                (int)smem));
+        // persistent grid: as many CTAs as fit at once, each striding over the tile list
+        const int per_sm = (int)((227 * 1024) / (smem + 1024));
+        uint64_t grid = (uint64_t)sm_count() * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
+        if (grid > need.tiles) grid = need.tiles ? need.tiles : 1;
+        timeline_tiles_kernel<<<(unsigned)grid, kTileThreads, smem, st>>>(ta);
+    }
+    profile_mark(st, false);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+
+    FinalArgs fa;
+    fa.lib = lv; fa.ps = ps; fa.slots = slots; fa.n_align = o->n_align; fa.walks = walks; fa.partials = partials;
+    fa.P_out = P_out; fa.evals_out = reinterpret_cast<unsigned long long*>(evals_out);
+    if (detail) fa.detail = *detail; else { roomie_pair_detail z = {}; fa.detail = z; }
+    finalize_kernel<<<ps.n_pairs, kFinalThreads, (size_t)slots * 2 * sizeof(float), st>>>(fa);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+    return ROOMIE_OK;
+}
+
+}  // namespace roomie
+
+using namespace roomie;
+
+extern "C" size_t roomie_pair_workspace_bytes(const roomie_library* lib, const roomie_opts* opts,
+                                              uint64_t pair_begin, uint64_t pair_end) {
+    if (check_lib(lib, opts) != ROOMIE_OK) return 0;
+    const uint64_t total = (uint64_t)lib->num_profiles * (lib->num_profiles + 1) / 2;
+    if (pair_end > total) pair_end = total;
+    if (pair_begin >= pair_end) return 0;
+    uint32_t slots;
+    if (slots_for(lib, opts, false, 0, 0, slots) != ROOMIE_OK) return 0;
+    Need need;
+    batch_need(lib, opts, false, 0, 0, pair_begin, pair_end, slots, need);
+    return bytes_for(need);
+}
+
+extern "C" int roomie_pair_matrix(const roomie_library* lib, const roomie_opts* opts, uint64_t pair_begin,
+                                  uint64_t pair_end, float* P_out, uint64_t* evals_out, void* workspace,
+                                  size_t workspace_bytes, void* stream) {
+    int rc = check_lib(lib, opts);
+    if (rc != ROOMIE_OK) return rc;
+    if (!P_out || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return ROOMIE_ERR_INVALID_ARG;
+    const uint64_t total = (uint64_t)lib->num_profiles * (lib->num_profiles + 1) / 2;
+    if (pair_end > total) pair_end = total;
+    if (pair_begin > pair_end) return ROOMIE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), st));
+    if (pair_begin == pair_end) return ROOMIE_OK;
+    uint32_t slots;
+    rc = slots_for(lib, opts, false, 0, 0, slots);
+    if (rc != ROOMIE_OK) return rc;
+
+    uint64_t p0 = pair_begin;
+    while (p0 < pair_end) {
+        // largest batch [p0, p1) whose scratch fits: try everything, then halve
+        uint64_t p1 = pair_end;
+        Need need;
+        for (;;) {
+            batch_need(lib, opts, false, 0, 0, p0, p1, slots, need);
+            if (bytes_for(need) <= workspace_bytes && need.walks < (1ull << 31) && need.tiles < (1ull << 31)) break;
+            if (p1 - p0 == 1) return ROOMIE_ERR_CAPACITY;
+            p1 = p0 + (p1 - p0) / 2;
+        }
+        PairSet ps;
+        ps.pair_begin = p0; ps.n_pairs = (uint32_t)(p1 - p0); ps.explicit_pair = 0; ps.a = ps.b = 0;
+        rc = run_batch(lib, opts, ps, slots, need, P_out, evals_out, nullptr, static_cast<unsigned char*>(workspace), st);
+        if (rc != ROOMIE_OK) return rc;
+        p0 = p1;
+    }
+    return ROOMIE_OK;
+}
+
+extern "C" int roomie_pair_interference(const roomie_library* lib, uint32_t a, uint32_t b, const roomie_opts* opts,
+                                        float* out2, uint64_t* evals_out, const roomie_pair_detail* detail,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_lib(lib, opts);
+    if (rc != ROOMIE_OK) return rc;
+    if (!out2 || !workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || a >= lib->num_profiles ||
+        b >= lib->num_profiles)
+        return ROOMIE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), st));
+    uint32_t slots;
+    rc = slots_for(lib, opts, true, a, b, slots);
+    if (rc != ROOMIE_OK) return rc;
+    Need need;
+    batch_need(lib, opts, true, a, b, 0, 1, slots, need);
+    if (bytes_for(need) > workspace_bytes) return ROOMIE_ERR_CAPACITY;
+    PairSet ps;
+    ps.pair_begin = 0; ps.n_pairs = 1; ps.explicit_pair = 1; ps.a = a; ps.b = b;
+    return run_batch(lib, opts, ps, slots, need, out2, evals_out, detail, static_cast<unsigned char*>(workspace), st);
+}

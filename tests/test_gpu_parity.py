@@ -1,0 +1,346 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Bar: occupancy integers, demand vectors, evaluation counts, kept alignments and placement
+indices bit-exact; float32 slowdowns within 1e-5 relative of the float64 oracle, and exactly 0
+where the oracle is 0."""
+import numpy as np
+import pytest
+
+import roomie_synth as rs
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def rm():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("gpu-marked test run without a CUDA device")
+    import paper_2607_16784_b200 as pkg
+    return pkg
+
+
+def to_np_u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def assert_close(got, want, rtol=RTOL):
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape
+    zero = want == 0
+    assert (got[zero] == 0).all()
+    err = np.abs(got - want)[~zero] / np.abs(want[~zero])
+    assert err.size == 0 or err.max() <= rtol, f"max rel err {err.max():.3e}"
+    return 0.0 if err.size == 0 else float(err.max())
+
+
+def build_both(rm, oracle, lib):
+    ol = oracle.library_build(lib)
+    gl = rm.library_build(lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block,
+                          lib.dur_us, lib.gap_us, lib.offsets, lib.spec)
+    return ol, gl
+
+
+# ----------------------------------------------------------------------------- occupancy
+@pytest.mark.parametrize("cfg", [0, 1, 2, 3, 4])
+def test_occupancy_bit_exact(rm, oracle, cfg):
+    for feasible in (True, False):
+        lib = rs.make_library(cfg, feasible=feasible)
+        if cfg == 3 and not feasible:
+            continue
+        want = oracle.occupancy(lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block, lib.spec)
+        got = rm.occupancy(lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block, lib.spec)
+        for name in ("b_lim", "b_res", "limiter", "warps"):
+            assert np.array_equal(got[name].cpu().numpy().astype(np.uint32), getattr(want, name)), name
+        assert np.array_equal(got["occ"].cpu().numpy().view(np.uint32), want.occ.view(np.uint32))
+        assert np.array_equal(got["occ_theo"].cpu().numpy().view(np.uint32), want.occ_theo.view(np.uint32))
+        assert np.array_equal(to_np_u32(got["phi"]), want.phi)
+        assert int(got["n_unlaunchable"].item()) == want.n_unlaunchable
+
+
+def test_occupancy_ragged_and_unaligned(rm, oracle):
+    lib = rs.make_library(1, feasible=False)
+    import torch
+    for n in (1, 3, 5, 1023, 1025):
+        # offset by one element: not 16-byte aligned -> scalar kernel; n % 4 != 0 -> scalar kernel
+        cols = [torch.from_numpy(np.ascontiguousarray(x[:n + 1]).view(np.int32)).cuda()[1:]
+                for x in (lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block)]
+        got = rm.occupancy(*cols, lib.spec)
+        want = oracle.occupancy(lib.grid_blocks[1:n + 1], lib.block_threads[1:n + 1],
+                                lib.regs_per_thread[1:n + 1], lib.smem_per_block[1:n + 1], lib.spec)
+        assert np.array_equal(got["b_res"].cpu().numpy().astype(np.uint32), want.b_res)
+        assert np.array_equal(to_np_u32(got["phi"]), want.phi)
+    empty = rm.occupancy([], [], [], [], lib.spec)
+    assert empty["occ"].numel() == 0
+
+
+def test_spec_out_of_range_is_rejected(rm):
+    with pytest.raises(rm.RoomieError):
+        rm.occupancy([1], [32], [8], [0], rs.GpuSpec(108, 1 << 18, 1024, 2048, 32))
+    with pytest.raises(rm.RoomieError):
+        rm.occupancy([1], [32], [8], [0], rs.GpuSpec(108, 65536, 1024, 2048, 256))
+
+
+# ----------------------------------------------------------------------------- timeline records
+@pytest.mark.parametrize("cfg", [0, 1, 2, 4])
+def test_library_records_bit_exact(rm, oracle, cfg):
+    lib = rs.make_library(cfg)
+    ol, gl = build_both(rm, oracle, lib)
+    rec = to_np_u32(gl.records)
+    assert np.array_equal(rec[:, 0], ol.start)
+    assert np.array_equal(rec[:, 1], ol.start + ol.dt)
+    phi = ol.occ.phi.astype(np.uint64)
+    assert np.array_equal(rec[:, 2], (phi[1] | (phi[0] << np.uint64(20))).astype(np.uint32))
+    assert np.array_equal(rec[:, 3], (phi[2] | (phi[3] << np.uint64(22))).astype(np.uint32))
+    assert np.array_equal(gl.T.cpu().numpy().view(np.uint64), ol.T)
+    assert gl.status_flags() == 0
+
+
+def test_library_range_flags(rm):
+    n = 30
+    one = np.ones(n, dtype=np.uint32)
+    gl = rm.library_build(one * 100, one * 64, one * 16, one * 0, np.full(n, 1e5, np.float32),
+                          np.zeros(n, np.float32), [0, n], rs.SPEC_CLOUD)
+    assert gl.status_flags() & 1                      # 30 x 1e8 ticks >= 2^31
+    gl = rm.library_build(one[:2], one[:2] * 64, one[:2] * 16, one[:2] * 0, np.array([-1.0, 1.0], np.float32),
+                          np.zeros(2, np.float32), [0, 2], rs.SPEC_CLOUD)
+    assert gl.status_flags() & 2
+
+
+# ----------------------------------------------------------------------------- pairwise walk
+SETTINGS = [dict(mode=0, n_align=1, start_filter=0), dict(mode=0, n_align=8, start_filter=1),
+            dict(mode=1, n_align=1, start_filter=0), dict(mode=1, n_align=8, start_filter=1)]
+
+
+def check_pair_detail(rm, oracle, ol, gl, a, b, **kw):
+    want = oracle.pair(ol, a, b, **kw)
+    cap = max(want.kept, 1)
+    got = rm.pair_interference(gl, a, b, detail_capacity=cap, **kw)
+    assert int(got["n_kept"].item()) == want.kept
+    k = want.kept
+    assert np.array_equal(to_np_u32(got["s_i"])[:k], want.s_i)
+    assert np.array_equal(to_np_u32(got["s_j"])[:k], want.s_j)
+    assert np.array_equal(to_np_u32(got["evals_c"])[:k].astype(np.uint64), want.evals_c)
+    assert np.array_equal(got["V"].cpu().numpy().view(np.uint64)[:k], want.V)
+    assert_close(got["delta_i"].cpu().numpy()[:k], want.delta_i)
+    assert_close(got["delta_j"].cpu().numpy()[:k], want.delta_j)
+    assert_close(got["P2"].cpu().numpy(), [want.P_ab, want.P_ba])
+    assert int(got["evals"].item()) == want.evals
+
+
+@pytest.mark.parametrize("kw", SETTINGS + [dict(mode=0, n_align=0, start_filter=0),
+                                           dict(mode=1, n_align=0, start_filter=1),
+                                           dict(mode=0, n_align=3, start_filter=1)])
+def test_config0_pair_detail(rm, oracle, kw):
+    for feasible in (True, False):
+        lib = rs.make_library(0, feasible=feasible)
+        ol, gl = build_both(rm, oracle, lib)
+        for a, b in ((0, 1), (1, 0), (0, 0), (1, 1)):
+            check_pair_detail(rm, oracle, ol, gl, a, b, **kw)
+
+
+def test_worked_example_on_gpu(rm):
+    """The hand-derived example of tests/golden/worked_example.txt, straight through the CUDA path."""
+    from test_oracle_walk import make_lib, read_example
+    prof, res = read_example()
+    X = [(int(a), int(b), int(c), int(d), e, g) for a, b, c, d, e, g in prof["X"]]
+    Y = [(int(a), int(b), int(c), int(d), e, g) for a, b, c, d, e, g in prof["Y"]]
+    lib = make_lib([X, Y])
+    gl = rm.library_build(lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block,
+                          lib.dur_us, lib.gap_us, lib.offsets, lib.spec)
+    for name, mode in (("TIMELINE", 0), ("LOCKSTEP", 1)):
+        ev, dx, dy, V, pxy, pyx = res[name]
+        got = rm.pair_interference(gl, 0, 1, mode=mode, detail_capacity=1)
+        assert int(got["evals"].item()) == int(ev)
+        assert float(got["delta_i"][0]) == dx * 1000 and float(got["delta_j"][0]) == dy * 1000
+        assert int(got["V"][0]) == int(V * 1000)
+        assert got["P2"].cpu().tolist() == [pxy, pyx]
+
+
+def test_ties_and_tiny_profiles(rm, oracle):
+    from test_oracle_walk import make_lib, tiny_lib
+    k = (256, 64, 0, 10000)
+    libs = [make_lib([[k + (0.004, 0.0)] * 3, [k + (0.006, 0.0)] * 2]),
+            make_lib([[k + (0.004, 0.0)] * 3, [k + (0.004, 0.0)] * 3]),
+            make_lib([[k + (0.004, 0.0)], [k + (0.004, 0.0)]]),
+            make_lib([[k + (0.002, 0.002)] * 40, [k + (0.004, 0.0)] * 21, [k + (0.001, 0.0)] * 1])]
+    libs += [tiny_lib(s, n_prof=3, qmax=9) for s in range(4)]
+    for lib in libs:
+        ol, gl = build_both(rm, oracle, lib)
+        P = ol.num_profiles
+        for a in range(P):
+            for b in range(P):
+                for kw in (dict(mode=0, n_align=0), dict(mode=0, n_align=2, start_filter=1), dict(mode=1, n_align=0)):
+                    check_pair_detail(rm, oracle, ol, gl, a, b, **kw)
+
+
+def test_many_ties_across_tile_boundaries(rm, oracle):
+    """Equal-duration zero-gap profiles: every step is a tie; several tiles and a ragged tail."""
+    from test_oracle_walk import make_lib
+    k1, k2 = (256, 64, 0, 10000, 0.005, 0.0), (128, 32, 49152, 10000, 0.005, 0.0)
+    rng = np.random.default_rng(0)
+    mk = lambda q: [k1 if rng.random() < 0.5 else k2 for _ in range(q)]
+    lib = make_lib([mk(3000), mk(4100), [k1[:4] + (0.010, 0.0)] * 1500])
+    ol, gl = build_both(rm, oracle, lib)
+    for a in range(3):
+        for b in range(3):
+            for kw in (dict(mode=0, n_align=1), dict(mode=0, n_align=5, start_filter=1), dict(mode=1, n_align=2)):
+                check_pair_detail(rm, oracle, ol, gl, a, b, **kw)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 4])
+@pytest.mark.parametrize("kw", SETTINGS)
+def test_pair_matrix_configs(rm, oracle, cfg, kw):
+    if cfg != 1 and kw["mode"] == 1 and kw["n_align"] == 1:
+        pytest.skip("lockstep is required on configs 0 and 1; one lockstep setting is kept for the others")
+    lib = rs.make_library(cfg)
+    ol, gl = build_both(rm, oracle, lib)
+    want, want_ev = oracle.pair_matrix(ol, **kw)
+    got, ev = rm.pair_matrix(gl, **kw)
+    assert int(ev.item()) == want_ev
+    assert_close(got.cpu().numpy(), want)
+    assert gl.status_flags() == 0
+
+
+def test_pair_matrix_ranges_and_batching(rm, oracle):
+    import torch
+    lib = rs.make_library(1)
+    ol, gl = build_both(rm, oracle, lib)
+    kw = dict(mode=0, n_align=8, start_filter=1)
+    full, ev_full = rm.pair_matrix(gl, **kw)
+    P = gl.num_profiles
+    total = P * (P + 1) // 2
+    # two disjoint ranges written into one matrix reproduce the full call bit for bit
+    out = torch.zeros_like(full)
+    _, e1 = rm.pair_matrix(gl, pair_begin=0, pair_end=37, out=out, **kw)
+    _, e2 = rm.pair_matrix(gl, pair_begin=37, pair_end=total, out=out, **kw)
+    assert torch.equal(out, full) and int(e1.item()) + int(e2.item()) == int(ev_full.item())
+    # a workspace far smaller than one batch forces many batches: same bits
+    small = torch.empty(rm.pair_workspace_bytes(gl, pair_begin=0, pair_end=3, **kw), dtype=torch.uint8, device="cuda")
+    out2, e3 = rm.pair_matrix(gl, workspace=small, **kw)
+    assert torch.equal(out2, full) and int(e3.item()) == int(ev_full.item())
+    # too small for a single pair -> CAPACITY
+    with pytest.raises(rm.RoomieError):
+        rm.pair_matrix(gl, workspace=torch.empty(512, dtype=torch.uint8, device="cuda"), **kw)
+    # empty range
+    z, e0 = rm.pair_matrix(gl, pair_begin=5, pair_end=5, **kw)
+    assert not z.any() and int(e0.item()) == 0
+    # single-pair entry point equals the matrix entries
+    for a, b in ((0, 0), (2, 9), (9, 2), (15, 15)):
+        p2 = rm.pair_interference(gl, a, b, **kw)["P2"].cpu().numpy()
+        assert p2[0] == full[a, b].item() and (a == b or p2[1] == full[b, a].item())
+
+
+def test_config3_full_size(rm, oracle):
+    """The headline workload in the launch configuration the benchmark times: full 512-profile matrix
+    at the base setting against the oracle, every entry; the greedy setting on a band of pairs."""
+    lib = rs.make_library(3)
+    ol, gl = build_both(rm, oracle, lib)
+    assert gl.status_flags() == 0
+    rec = to_np_u32(gl.records)
+    assert np.array_equal(rec[:, 0], ol.start) and np.array_equal(rec[:, 1], ol.start + ol.dt)
+    want, want_ev = oracle.pair_matrix(ol, mode=0, n_align=1, start_filter=0)
+    got, ev = rm.pair_matrix(gl, mode=0, n_align=1, start_filter=0)
+    assert int(ev.item()) == want_ev
+    assert_close(got.cpu().numpy(), want)
+    # greedy setting: pairs 40 000 .. 40 600 of the triangle
+    import torch
+    lo, hi = 40000, 40600
+    wantg, wev = oracle.pair_matrix(ol, mode=0, n_align=8, start_filter=1, pair_begin=lo, pair_end=hi)
+    gotg, gev = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1, pair_begin=lo, pair_end=hi)
+    assert int(gev.item()) == wev
+    assert_close(gotg.cpu().numpy(), wantg)
+    assert gl.status_flags() == 0
+
+
+# ----------------------------------------------------------------------------- estimate + placement
+def test_multi_estimate_bit_exact(rm, oracle):
+    rng = np.random.default_rng(1)
+    P, R, n = 40, 8, 300
+    Pm = rng.random((P, P)).astype(np.float32)
+    ids = rng.integers(0, P, (n, R)).astype(np.int32)
+    cnt = rng.integers(0, R + 1, n).astype(np.uint32)
+    inc = rng.integers(0, P, n).astype(np.int32)
+    mu, mean = rm.multi_estimate(Pm, ids, cnt, inc, max_residents=R)
+    mu, mean = mu.cpu().numpy(), mean.cpu().numpy()
+    for s in range(n):
+        wmu, wmean, _, _ = oracle.multi_estimate(Pm, ids[s, :cnt[s]], inc[s])
+        assert np.array_equal(mu[s, :cnt[s] + 1].view(np.uint32), wmu.view(np.uint32))
+        assert mean[s].view(np.uint32) == np.float32(wmean).view(np.uint32)
+
+
+def run_place(rm, oracle, Pm32, cl, lam):
+    st = rm.ClusterState(cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0)
+    gpu, mean, mu_arr = rm.place(Pm32, st, cl.arr_id, cl.arr_life, lam)
+    want = oracle.place(Pm32, cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0,
+                        cl.arr_id, cl.arr_life, lam)
+    return st, gpu.cpu().numpy(), mean.cpu().numpy(), mu_arr.cpu().numpy(), want
+
+
+@pytest.mark.parametrize("cfg", [2, 4])
+def test_placement_same_matrix_bit_exact(rm, oracle, cfg):
+    """Protocol 1: oracle and GPU are fed the same float32 matrix -> every decision identical."""
+    lib = rs.make_library(cfg)
+    cl = rs.make_cluster(cfg)
+    ol, gl = build_both(rm, oracle, lib)
+    Pm, _ = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)
+    Pm32 = Pm.cpu().numpy()
+    for lam in (cl.lam, 0.25, 1e9):
+        st, gpu, mean, mu_arr, want = run_place(rm, oracle, Pm32, cl, lam)
+        assert np.array_equal(gpu, want.gpu)
+        assert np.array_equal(mean.view(np.uint32), want.mean.view(np.uint32))
+        assert np.array_equal(mu_arr.view(np.uint32), want.mu_arr.view(np.uint32))
+        assert np.array_equal(st.ids.cpu().numpy(), want.ids)
+        assert np.array_equal(to_np_u32(st.expiry), want.expiry)
+        assert np.array_equal(to_np_u32(st.count), want.count)
+        assert int(st.tick.item()) == want.tick == len(cl.arr_id)
+    assert (want.gpu >= 0).any()
+
+
+@pytest.mark.parametrize("cfg", [2, 4])
+def test_placement_end_to_end(rm, oracle, cfg):
+    """Protocol 2: GPU matrix vs oracle matrix.  A decision may differ only where the oracle's double
+    shadow shows a near-tie; after the first such difference the states diverge, so only the prefix
+    up to it is compared."""
+    lib = rs.make_library(cfg)
+    cl = rs.make_cluster(cfg)
+    ol, gl = build_both(rm, oracle, lib)
+    Pg, _ = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)
+    Po, _ = oracle.pair_matrix(ol, mode=0, n_align=8, start_filter=1)
+    st = rm.ClusterState(cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0)
+    gpu = rm.place(Pg, st, cl.arr_id, cl.arr_life, cl.lam)[0].cpu().numpy()
+    want = oracle.place(Po.astype(np.float32), cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0,
+                        cl.arr_id, cl.arr_life, cl.lam)
+    diff = np.nonzero(gpu != want.gpu)[0]
+    if diff.size:
+        assert want.near_tie[diff[0]], f"first mismatch at arrival {diff[0]} is not a near-tie"
+    print(f"\n[placement cfg{cfg}] mismatching decisions before divergence: {0 if not diff.size else 1}")
+
+
+def test_placement_edge_cases(rm, oracle):
+    Pm = np.full((3, 3), 0.25, dtype=np.float32)
+    cases = [
+        (4, 2, [-1] * 8, [0] * 4, [0, 1, 2, 0, 1], [0] * 5, 0.5),
+        (2, 2, [-1] * 4, [0, 0], [0] * 6, [0] * 6, 1e9),
+        (1, 1, [-1], [0], [0] * 4, [1] * 4, 0.5),
+        (1, 1, [-1], [0], [0] * 4, [2] * 4, 0.5),
+        (33, 3, [-1] * 99, [0] * 33, list(range(3)) * 40, [5] * 120, 0.3),
+    ]
+    for G, R, ids, count, aid, life, lam in cases:
+        st = rm.ClusterState(G, R, ids, [0] * (G * R), count, 7)
+        gpu = rm.place(Pm, st, aid, life, lam)[0].cpu().numpy()
+        want = oracle.place(Pm, G, R, ids, [0] * (G * R), count, 7, aid, life, lam)
+        assert np.array_equal(gpu, want.gpu)
+        assert np.array_equal(st.ids.cpu().numpy(), want.ids) and int(st.tick.item()) == want.tick
+    # matrix too large for shared memory -> read from global memory: same decisions
+    rng = np.random.default_rng(5)
+    P = 300
+    big = (rng.random((P, P)) * 0.3).astype(np.float32)
+    cl = rs.make_cluster(2, num_profiles=P, num_arrivals=500)
+    st = rm.ClusterState(cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0)
+    gpu = rm.place(big, st, cl.arr_id, cl.arr_life, 0.5)[0].cpu().numpy()
+    want = oracle.place(big, cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0, cl.arr_id, cl.arr_life, 0.5)
+    assert np.array_equal(gpu, want.gpu)
