@@ -108,9 +108,10 @@ typedef struct roomie_library {
     roomie_gpu_spec spec;
 } roomie_library;
 
-/* Number of floats of roomie_library.share_table for a spec: 2 * (W+1)^2, W = threads_per_sm/32.
- * Entry (wa, wb) holds {wa/(wa+wb), wb/(wa+wb)}: the occupancy shares o_i/(o_i+o_j) of
- * Algorithm 1 line 13 (W cancels). */
+/* Number of floats of roomie_library.share_table for a spec: 2W + 1, W = threads_per_sm/32.
+ * Entry s holds 1/s (entry 0 is 0): the occupancy share o_i/(o_i+o_j) of Algorithm 1 line 13
+ * equals warps_i * table[warps_i + warps_j] (W cancels); a charged delay is evaluated as
+ * (ticks * table[...]) * warps_i in float32. */
 size_t roomie_share_table_floats(const roomie_gpu_spec *spec /* host */);
 
 /* Builds the library from a kernel table plus isolated durations and inter-kernel gaps

@@ -159,17 +159,11 @@ __global__ void __launch_bounds__(kBuildThreads) library_build_kernel(BuildArgs 
     if (threadIdx.x == 0) a.T[m] = sum_d;
 }
 
-// Occupancy shares o_i/(o_i+o_j) = warps_i/(warps_i+warps_j) for every pair of warp counts.
-__global__ void share_table_kernel(float2* tab, uint32_t Wt) {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= Wt * Wt) return;
-    const uint32_t wa = i / Wt, wb = i % Wt;
-    float2 v = make_float2(0.0f, 0.0f);
-    if (wa + wb) {
-        v.x = __fdiv_rn((float)wa, (float)(wa + wb));
-        v.y = __fdiv_rn((float)wb, (float)(wa + wb));
-    }
-    tab[i] = v;
+// Reciprocals 1/s for every possible sum of two warp counts: the occupancy share of
+// Algorithm 1 line 13 is o_i/(o_i+o_j) = warps_i * (1 / (warps_i + warps_j)).
+__global__ void share_table_kernel(float* tab, uint32_t n) {
+    const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < n) tab[s] = s ? __frcp_rn((float)s) : 0.0f;
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -217,8 +211,7 @@ extern "C" int roomie_occupancy(const roomie_kernel_table* table, const roomie_g
 
 extern "C" size_t roomie_share_table_floats(const roomie_gpu_spec* spec) {
     if (validate_spec(spec) != ROOMIE_OK) return 0;
-    const size_t Wt = spec->threads_per_sm / 32u + 1u;
-    return 2 * Wt * Wt;
+    return 2 * (size_t)(spec->threads_per_sm / 32u) + 1u;
 }
 
 extern "C" int roomie_library_build(const roomie_library* lib, const roomie_kernel_table* table,
@@ -248,8 +241,8 @@ extern "C" int roomie_library_build(const roomie_library* lib, const roomie_kern
     library_build_kernel<<<lib->num_profiles, kBuildThreads, 0, st>>>(a);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
-    const uint32_t Wt = lib->spec.threads_per_sm / 32u + 1u;
-    share_table_kernel<<<(Wt * Wt + 255) / 256, 256, 0, st>>>(reinterpret_cast<float2*>(lib->share_table), Wt);
+    const uint32_t n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u;
+    share_table_kernel<<<(n_inv + 255) / 256, 256, 0, st>>>(lib->share_table, n_inv);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;

@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(256) plan_kernel(PlanArgs g) {
     const int lane = threadIdx.x & 31;
     bool valid = w < n_walks;
     uint32_t a = 0, b = 0, offa = 0, offb = 0, si = 0, sj = 0, na = 0, nb = 0, baseA = 0, baseB = 0;
-    uint32_t L = 0, n_tiles = 0;
+    uint32_t L = 0, n_tiles = 0, final_tie = 0;
     const uint4 *RA = nullptr, *RB = nullptr;
     if (valid) {
         const uint32_t local = (uint32_t)(w / g.slots), c = (uint32_t)(w % g.slots);
@@ -126,6 +126,10 @@ __global__ void __launch_bounds__(256) plan_kernel(PlanArgs g) {
                         if (__ldg(&RB[mid].y) - baseB < endA) lo = mid + 1; else hi = mid;
                     }
                     L = na + lo;
+                    // the tile kernel counts every state with equal end times as a tie; the walk's
+                    // last state is one when A's last kernel ends together with a B kernel, but no
+                    // intermediate state follows it, so it is given back here
+                    if (lo < nb && __ldg(&RB[lo].y) - baseB == endA) final_tie = 1;
                 } else {                     // B runs out first: A kernels ending at or before
                     uint32_t lo = 0, hi = na;
                     while (lo < hi) {
@@ -151,7 +155,7 @@ __global__ void __launch_bounds__(256) plan_kernel(PlanArgs g) {
     base = __shfl_sync(0xffffffffu, base, 31) + incl - n_tiles;
     if (w < n_walks) {
         WalkInfo wi;
-        wi.tile_base = base; wi.n_tiles = n_tiles; wi.length = L; wi.valid = valid ? 1u : 0u;
+        wi.tile_base = base; wi.n_tiles = n_tiles; wi.length = L + final_tie; wi.valid = valid ? 1u : 0u;
         g.walks[w] = wi;
     }
     if (!valid || n_tiles == 0) return;
@@ -201,11 +205,23 @@ struct TileArgs {
     const uint32_t* tile_counter;
     uint32_t tile_capacity;
     TilePartial* partials;
-    const float2* share_table;
-    uint32_t Wt;                 // W + 1
+    const float* inv_table;      // [2W + 1] 1/s
+    uint32_t n_inv;              // 2W + 1
     PhiCap cap;
 };
 
+// Shared-memory layout of one tile.  Records are padded by one slot after every 8 so that the
+// lanes of a warp, whose positions on the merge path are about 8 records apart, fall into
+// different bank groups; the search keys (end ticks, re-based) live in their own array with
+// one pad word per 32 so that the binary-search probes of a warp do not collide either.
+__device__ __forceinline__ uint32_t rec_slot(uint32_t i) { return i + (i >> 3); }
+__device__ __forceinline__ uint32_t key_slot(uint32_t i) { return i + (i >> 5); }
+constexpr int kTileLoad = kTileItems + 2;                               // one look-ahead record per side
+constexpr int kRecSlots = kTileLoad + (kTileLoad >> 3) + 2;
+constexpr int kKeySlots = kTileLoad + (kTileLoad >> 5) + 2;
+constexpr int kStageBatch = 6;                                           // global loads in flight per thread
+
+template <bool kWithV>
 __device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned long long V, uint32_t ties,
                                                    TilePartial* out, float* s_f, unsigned long long* s_v,
                                                    uint32_t* s_t, int nwarps) {
@@ -213,7 +229,7 @@ __device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned 
     for (int s = 16; s > 0; s >>= 1) {
         di += __shfl_xor_sync(0xffffffffu, di, s);
         dj += __shfl_xor_sync(0xffffffffu, dj, s);
-        V += __shfl_xor_sync(0xffffffffu, V, s);
+        if (kWithV) V += __shfl_xor_sync(0xffffffffu, V, s);
         ties += __shfl_xor_sync(0xffffffffu, ties, s);
     }
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -227,67 +243,90 @@ __device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned 
     }
 }
 
-__global__ void __launch_bounds__(kTileThreads) timeline_tiles_kernel(TileArgs g) {
+// float of a small non-negative integer without the conversion unit
+__device__ __forceinline__ float small_int_to_float(uint32_t v) {
+    return __uint_as_float(0x4B000000u | v) - 8388608.0f;
+}
+
+template <bool kWithV>
+__global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArgs g) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float2* s_tab = reinterpret_cast<float2*>(smem_raw);
-    uint4* s_rec = reinterpret_cast<uint4*>(smem_raw + (((size_t)g.Wt * g.Wt * sizeof(float2) + 15) & ~(size_t)15));
+    uint4* s_rec = reinterpret_cast<uint4*>(smem_raw);
+    int32_t* s_key = reinterpret_cast<int32_t*>(smem_raw + (size_t)kRecSlots * sizeof(uint4));
+    float* s_inv = reinterpret_cast<float*>(s_key + kKeySlots);
     __shared__ float s_f[2 * kTileThreads / 32];
     __shared__ unsigned long long s_v[kTileThreads / 32];
     __shared__ uint32_t s_t[kTileThreads / 32];
 
-    for (uint32_t i = threadIdx.x; i < g.Wt * g.Wt; i += kTileThreads) s_tab[i] = __ldg(&g.share_table[i]);
+    for (uint32_t i = threadIdx.x; i < g.n_inv; i += kTileThreads) s_inv[i] = __ldg(&g.inv_table[i]);
     const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
 
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
         const TileDesc d = g.tiles[t];
         const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
+        const uint32_t n_load = loadA + loadB;
         __syncthreads();                                   // previous tile fully consumed
-        for (uint32_t i = threadIdx.x; i < loadA + loadB; i += kTileThreads)
-            s_rec[i] = __ldg(i < loadA ? &g.records[d.recA + i] : &g.records[d.recB + (i - loadA)]);
+        // stage the tile: A records first, then B; ticks re-based to the alignment's start
+        for (uint32_t i0 = threadIdx.x; i0 < n_load; i0 += kTileThreads * kStageBatch) {
+            uint4 r[kStageBatch];
+#pragma unroll
+            for (int j = 0; j < kStageBatch; ++j) {
+                const uint32_t i = i0 + j * kTileThreads;
+                if (i < n_load) r[j] = __ldg(i < loadA ? &g.records[d.recA + i] : &g.records[d.recB + (i - loadA)]);
+            }
+#pragma unroll
+            for (int j = 0; j < kStageBatch; ++j) {
+                const uint32_t i = i0 + j * kTileThreads;
+                if (i < n_load) {
+                    const uint32_t base = i < loadA ? d.baseA : d.baseB;
+                    r[j].x -= base; r[j].y -= base;
+                    s_rec[rec_slot(i)] = r[j];
+                    s_key[key_slot(i)] = (int32_t)r[j].y;
+                }
+            }
+        }
         __syncthreads();
-        const uint4* sA = s_rec;
-        const uint4* sB = s_rec + loadA;
         const uint32_t len = d.cntA + d.cntB;
         const uint32_t diag = threadIdx.x * kItems;
         float di = 0.0f, dj = 0.0f;
         unsigned long long V = 0;
         uint32_t ties = 0;
         if (diag < len) {
-            // this thread's start point on the tile's merge path
+            // this thread's start point on the tile's merge path (A first on equal end times)
             uint32_t lo = diag > d.cntB ? diag - d.cntB : 0u, hi = diag < d.cntA ? diag : d.cntA;
             while (lo < hi) {
                 const uint32_t mid = (lo + hi) >> 1;
-                if (sA[mid].y - d.baseA <= sB[diag - 1 - mid].y - d.baseB) lo = mid + 1; else hi = mid;
+                if (s_key[key_slot(mid)] <= s_key[key_slot(loadA + diag - 1 - mid)]) lo = mid + 1; else hi = mid;
             }
-            uint32_t x = lo, y = diag - lo;
+            uint32_t x = lo, y = loadA + diag - lo;                   // unified record indices
             const uint32_t steps = (len - diag < (uint32_t)kItems) ? len - diag : (uint32_t)kItems;
-            const uint32_t tie_limit = d.cntA + (d.flags & 1u);     // x + 1 < tie_limit: A has a next kernel
-            uint4 ra = sA[x], rb = sB[y];
-            int32_t Sa = (int32_t)(ra.x - d.baseA), Ea = (int32_t)(ra.y - d.baseA);
-            int32_t Sb = (int32_t)(rb.x - d.baseB), Eb = (int32_t)(rb.y - d.baseB);
+            uint4 ra = s_rec[rec_slot(x)], rb = s_rec[rec_slot(y)];
+            uint32_t slack_lo = g.cap.lo - ra.z, slack_hi = g.cap.hi - ra.w;
+            uint32_t wa = ra.z >> kWarpShift, wb = rb.z >> kWarpShift;
+            float fa = small_int_to_float(wa), fb = small_int_to_float(wb);
 #pragma unroll
             for (int s = 0; s < kItems; ++s) {
                 if ((uint32_t)s < steps) {
-                    const int32_t ov = min(Ea, Eb) - max(Sa, Sb);
-                    const bool hit = (ov > 0) && phi_exceeds(g.cap.lo - ra.z, g.cap.hi - ra.w, rb.z, rb.w);
-                    const float2 w = s_tab[(ra.z >> kWarpShift) * g.Wt + (rb.z >> kWarpShift)];
-                    const float ovf = hit ? (float)ov : 0.0f;
-                    di = fmaf(ovf, w.x, di);
-                    dj = fmaf(ovf, w.y, dj);
-                    V += hit ? (unsigned long long)(uint32_t)ov : 0ull;
-                    const bool adv_a = Ea <= Eb;
-                    ties += (Ea == Eb && x + 1 < tie_limit) ? 1u : 0u;
-                    if (adv_a) {
-                        ++x; ra = sA[x];
-                        Sa = (int32_t)(ra.x - d.baseA); Ea = (int32_t)(ra.y - d.baseA);
+                    const int32_t Ea = (int32_t)ra.y, Eb = (int32_t)rb.y;
+                    const int32_t ov = min(Ea, Eb) - max((int32_t)ra.x, (int32_t)rb.x);
+                    const bool hit = (ov > 0) && phi_exceeds(slack_lo, slack_hi, rb.z, rb.w);
+                    const float tw = (hit ? (float)ov : 0.0f) * s_inv[wa + wb];   // overlap / (o_i + o_j)
+                    di = fmaf(tw, fa, di);
+                    dj = fmaf(tw, fb, dj);
+                    if (kWithV) V += hit ? (unsigned long long)(uint32_t)ov : 0ull;
+                    ties += (Ea == Eb) ? 1u : 0u;
+                    if (Ea <= Eb) {
+                        ++x; ra = s_rec[rec_slot(x)];
+                        slack_lo = g.cap.lo - ra.z; slack_hi = g.cap.hi - ra.w;
+                        wa = ra.z >> kWarpShift; fa = small_int_to_float(wa);
                     } else {
-                        ++y; rb = sB[y];
-                        Sb = (int32_t)(rb.x - d.baseB); Eb = (int32_t)(rb.y - d.baseB);
+                        ++y; rb = s_rec[rec_slot(y)];
+                        wb = rb.z >> kWarpShift; fb = small_int_to_float(wb);
                     }
                 }
             }
         }
-        block_reduce_store(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
+        block_reduce_store<kWithV>(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
     }
 }
 
@@ -306,15 +345,16 @@ __global__ void __launch_bounds__(kTileThreads) lockstep_tiles_kernel(TileArgs g
         for (uint32_t i = threadIdx.x; i < d.cntA; i += kTileThreads) {
             const uint4 ra = __ldg(&g.records[d.recA + i]), rb = __ldg(&g.records[d.recB + i]);
             if (phi_exceeds(g.cap.lo - ra.z, g.cap.hi - ra.w, rb.z, rb.w)) {
-                const float2 w = __ldg(&g.share_table[(ra.z >> kWarpShift) * g.Wt + (rb.z >> kWarpShift)]);
+                const uint32_t wa = ra.z >> kWarpShift, wb = rb.z >> kWarpShift;
+                const float inv = __ldg(&g.inv_table[wa + wb]);
                 const uint32_t da = ra.y - ra.x, db = rb.y - rb.x;
-                di = fmaf((float)da, w.x, di);
-                dj = fmaf((float)db, w.y, dj);
+                di = fmaf((float)da * inv, small_int_to_float(wa), di);
+                dj = fmaf((float)db * inv, small_int_to_float(wb), dj);
                 V += (unsigned long long)da + db;
             }
         }
         __syncthreads();
-        block_reduce_store(di, dj, V, 0u, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
+        block_reduce_store<true>(di, dj, V, 0u, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
     }
 }
 
@@ -554,25 +594,25 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
 
     TileArgs ta;
     ta.records = lv.records; ta.tiles = tiles; ta.tile_counter = counter; ta.tile_capacity = (uint32_t)need.tiles; ta.partials = partials;
-    ta.share_table = reinterpret_cast<const float2*>(lib->share_table);
-    ta.Wt = lib->spec.threads_per_sm / 32u + 1u; ta.cap = lv.cap;
+    ta.inv_table = lib->share_table;
+    ta.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u; ta.cap = lv.cap;
     profile_mark(st, true);
     if (pa.lockstep) {
         uint64_t grid = (uint64_t)sm_count() * 8;
         if (grid > need.tiles) grid = need.tiles ? need.tiles : 1;
         lockstep_tiles_kernel<<<(unsigned)grid, kTileThreads, 0, st>>>(ta);
     } else {
-        const size_t tab = ((size_t)ta.Wt * ta.Wt * sizeof(float2) + 15) & ~(size_t)15;
-        const size_t smem = tab + (size_t)(kTileItems + 4) * sizeof(uint4);
-        if (smem > 227 * 1024) return ROOMIE_ERR_CAPACITY;
+        const size_t smem = (size_t)kRecSlots * sizeof(uint4) + (size_t)kKeySlots * sizeof(int32_t) +
+                            (size_t)ta.n_inv * sizeof(float);
+        auto kern = detail ? timeline_tiles_kernel<true> : timeline_tiles_kernel<false>;
         if (smem > 48 * 1024)
-            ROOMIE_CUDA_OK(cudaFuncSetAttribute(timeline_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                (int)smem));
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         // persistent grid: as many CTAs as fit at once, each striding over the tile list
-        const int per_sm = (int)((227 * 1024) / (smem + 1024));
-        uint64_t grid = (uint64_t)sm_count() * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
+        int per_sm = (int)((227 * 1024) / (smem + 1024 + 256));
+        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
+        uint64_t grid = (uint64_t)sm_count() * per_sm;
         if (grid > need.tiles) grid = need.tiles ? need.tiles : 1;
-        timeline_tiles_kernel<<<(unsigned)grid, kTileThreads, smem, st>>>(ta);
+        kern<<<(unsigned)grid, kTileThreads, smem, st>>>(ta);
     }
     profile_mark(st, false);
     note_launch();

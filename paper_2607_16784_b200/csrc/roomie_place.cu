@@ -35,9 +35,20 @@ __global__ void __launch_bounds__(128) multi_estimate_kernel(const float* __rest
 
 // ---------------------------------------------------------------------------------------
 // K5: the arrival stream is a dependent chain (each decision changes the state the next one
-// sees), so one CTA walks it with one thread per modelled GPU.  Per GPU and resident the sum
-// over the other residents is cached (`partial`); adding the arrival's term last reproduces
-// the slot-order float32 sum exactly, so a what-if costs 2 matrix reads per resident.
+// sees), so one CTA walks it with one thread per modelled GPU and the whole state in shared
+// memory.  What keeps the chain short:
+//   - per GPU and resident, the sum over the other residents is cached (`partial`); adding the
+//     arrival's term last reproduces the slot-order float32 sum exactly, so a what-if costs two
+//     matrix reads per resident;
+//   - the matrix row and column of the arrivals two steps ahead are fetched into a 4-deep
+//     shared-memory ring with cp.async while the current arrival is scored (or the whole matrix
+//     sits in shared memory when it fits);
+//   - the pairwise terms between the residents of a GPU are kept in shared memory, so that a
+//     departure re-sums the cached values without touching the matrix;
+//   - one barrier per arrival: warp argmin by two redux steps, cross-warp through a
+//     double-buffered slot array.
+// State arrays are slot-major in shared memory (slot * G + gpu) so that the threads of a warp
+// touch consecutive banks.
 // ---------------------------------------------------------------------------------------
 struct PlaceArgs {
     const float* Pm;
@@ -54,126 +65,223 @@ struct PlaceArgs {
     int32_t* gpu_out;
     float* mean_out;
     float* mu_arr_out;
-    int matrix_in_smem;
+    int matrix_mode;        // 0: whole matrix in shared memory, 1: row/column ring, 2: global loads
+    int pair_cache;         // 1: resident-resident terms cached in shared memory ([R][R][G] floats)
 };
 
 constexpr unsigned long long kNoGpu = ~0ull;
+constexpr uint32_t kArrChunk = 1024;      // arrivals staged in shared memory at a time
+constexpr int kRing = 4;      // arrival k+2 is fetched while k is scored and k-1's winner still reads its column
 
-__device__ __forceinline__ void recompute_partials(const float* Pm, uint32_t P, const int32_t* ids, float* partial,
-                                                   uint32_t c) {
-    for (uint32_t t = 0; t < c; ++t) {
-        const float* row = Pm + (size_t)ids[t] * P;
-        float s = 0.0f;
-        for (uint32_t u = 0; u < c; ++u)
-            if (u != t) s = __fadd_rn(s, row[ids[u]]);
-        partial[t] = s;
-    }
+__device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gmem_src) {
+    const uint32_t s = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(kPending) : "memory"); }
 
+// kSlots > 0: compile-time bound of the per-GPU slot loops (fully unrolled, predicated), R <= kSlots;
+// kSlots = 0: plain loops for any R
+template <int kSlots>
 __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const uint32_t GR = g.G * g.R;
+    const uint32_t G = g.G, R = g.R, P = g.P, GR = G * R;
     int32_t* s_ids = reinterpret_cast<int32_t*>(smem_raw);
     uint32_t* s_exp = reinterpret_cast<uint32_t*>(s_ids + GR);
     float* s_part = reinterpret_cast<float*>(s_exp + GR);
-    float* s_P = s_part + GR;
+    int32_t* s_arr = reinterpret_cast<int32_t*>(s_part + GR);       // [2][kArrChunk] ids, lifetimes
+    float* s_pair = reinterpret_cast<float*>(s_arr + 2 * kArrChunk); // [R][R][G] terms between residents
+    float* s_mat = s_pair + (g.pair_cache ? (size_t)GR * R : 0);     // mode 0: P*P, mode 1: ring [kRing][2][P]
     __shared__ unsigned long long s_key[2][32];
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = blockDim.x >> 5;
-    const float* Pm = g.Pm;
-    if (g.matrix_in_smem) {
-        for (uint32_t i = tid; i < g.P * g.P; i += blockDim.x) s_P[i] = g.Pm[i];
-        Pm = s_P;
+    const float* __restrict__ Pm = g.Pm;
+    if (g.matrix_mode == 0)
+        for (uint32_t i = tid; i < P * P; i += blockDim.x) s_mat[i] = Pm[i];
+    for (uint32_t i = tid; i < GR; i += blockDim.x) {                 // [gpu][slot] -> [slot][gpu]
+        const uint32_t gpu = i / R, slot = i % R;
+        s_ids[slot * G + gpu] = g.ids[i];
+        s_exp[slot * G + gpu] = g.expiry[i];
     }
-    for (uint32_t i = tid; i < GR; i += blockDim.x) { s_ids[i] = g.ids[i]; s_exp[i] = g.expiry[i]; }
     __syncthreads();
 
-    const bool owner = tid < g.G;
-    int32_t* my_ids = s_ids + (size_t)tid * g.R;
-    uint32_t* my_exp = s_exp + (size_t)tid * g.R;
-    float* my_part = s_part + (size_t)tid * g.R;
+    const bool owner = tid < G;
+    auto ID = [&](uint32_t t) -> int32_t& { return s_ids[t * G + tid]; };
+    auto EX = [&](uint32_t t) -> uint32_t& { return s_exp[t * G + tid]; };
+    auto PA = [&](uint32_t t) -> float& { return s_part[t * G + tid]; };
+    // element (i, j) of the matrix for bookkeeping off the fast path
+    auto mat = [&](int32_t i, int32_t j) -> float {
+        return g.matrix_mode == 0 ? s_mat[(size_t)i * P + j] : __ldg(&Pm[(size_t)i * P + j]);
+    };
+    auto PT = [&](uint32_t t, uint32_t u) -> float& { return s_pair[(t * R + u) * G + tid]; };   // P[id_t][id_u]
+    auto recompute_partials = [&](uint32_t c) {
+        for (uint32_t t = 0; t < c; ++t) {
+            float s = 0.0f;
+            for (uint32_t u = 0; u < c; ++u)
+                if (u != t) s = __fadd_rn(s, g.pair_cache ? PT(t, u) : mat(ID(t), ID(u)));
+            PA(t) = s;
+        }
+    };
     uint32_t c = 0, next_exp = 0xffffffffu;
     if (owner) {
-        c = min(g.count[tid], g.R);
-        recompute_partials(Pm, g.P, my_ids, my_part, c);
+        c = min(g.count[tid], R);
+        if (g.pair_cache)
+            for (uint32_t t = 0; t < c; ++t)
+                for (uint32_t u = 0; u < c; ++u) PT(t, u) = mat(ID(t), ID(u));
+        recompute_partials(c);
         for (uint32_t s = 0; s < c; ++s)
-            if (my_exp[s] && my_exp[s] < next_exp) next_exp = my_exp[s];
+            if (EX(s) && EX(s) < next_exp) next_exp = EX(s);
     }
     const uint32_t tick0 = *g.tick;
 
-    for (uint32_t k = 0; k < g.n; ++k) {
-        const uint32_t now = tick0 + k;
-        const int32_t inc = __ldg(&g.arr_id[k]);
-        unsigned long long key = kNoGpu;
-        float mean = 0.0f, mu_inc = 0.0f;
-        if (owner) {
-            if (next_exp <= now) {                       // departures, order kept
-                uint32_t w = 0;
-                next_exp = 0xffffffffu;
-                for (uint32_t s = 0; s < c; ++s) {
-                    const uint32_t e = my_exp[s];
-                    if (e != 0 && e <= now) continue;
-                    my_ids[w] = my_ids[s]; my_exp[w] = e;
-                    if (e && e < next_exp) next_exp = e;
-                    ++w;
-                }
-                for (uint32_t s = w; s < c; ++s) { my_ids[s] = -1; my_exp[s] = 0; }
-                c = w;
-                recompute_partials(Pm, g.P, my_ids, my_part, c);
-            }
-            if (c < g.R) {                                // what-if: residents + the arrival
-                const float* row_inc = Pm + (size_t)inc * g.P;
-                float tot = 0.0f;
-                for (uint32_t t = 0; t < c; ++t) {
-                    const int32_t id = my_ids[t];
-                    const float mu_t = __fadd_rn(my_part[t], Pm[(size_t)id * g.P + inc]);
-                    tot = __fadd_rn(tot, mu_t);
-                    mu_inc = __fadd_rn(mu_inc, row_inc[id]);
-                }
-                tot = __fadd_rn(tot, mu_inc);
-                mean = __fdiv_rn(tot, (float)(c + 1));
-                if (mean < g.lambda)                      // Algorithm 2 line 7; mean >= 0 so its bits order
-                    key = ((unsigned long long)__float_as_uint(mean) << 32) | tid;
-            }
+    // ring prefetch of row inc (P[inc][*]) and column inc (P[*][inc]) of arrival k
+    auto prefetch = [&](uint32_t k, int32_t inc) {
+        float* row = s_mat + (size_t)(k % kRing) * 2 * P;
+        float* col = row + P;
+        for (uint32_t i = tid; i < P; i += blockDim.x) {
+            cp_async_4(row + i, Pm + (size_t)inc * P + i);
+            cp_async_4(col + i, Pm + (size_t)i * P + inc);
         }
-        // argmin over GPUs, lowest index on equal means
-        unsigned long long best = key;
-#pragma unroll
-        for (int s = 16; s > 0; s >>= 1) {
-            const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, s);
-            best = o < best ? o : best;
-        }
-        if (lane == 0) s_key[k & 1][wid] = best;
+    };
+
+    for (uint32_t k0 = 0; k0 < g.n; k0 += kArrChunk) {
+        const uint32_t kn = min(kArrChunk, g.n - k0);
         __syncthreads();
-        best = s_key[k & 1][0];
-        for (uint32_t w = 1; w < nwarps; ++w) {
-            const unsigned long long o = s_key[k & 1][w];
-            best = o < best ? o : best;
+        for (uint32_t i = tid; i < kn; i += blockDim.x) {
+            s_arr[i] = g.arr_id[k0 + i];
+            s_arr[kArrChunk + i] = (int32_t)g.arr_life[k0 + i];
         }
-        if (best == kNoGpu) {
-            if (tid == 0) {
-                g.gpu_out[k] = -1;
-                if (g.mean_out) g.mean_out[k] = 0.0f;
-                if (g.mu_arr_out) g.mu_arr_out[k] = 0.0f;
+        __syncthreads();
+        if (g.matrix_mode == 1) {                                      // prime the ring: arrivals 0 and 1
+            prefetch(0, s_arr[0]);
+            cp_async_commit();
+            if (kn > 1) prefetch(1, s_arr[1]);
+            cp_async_commit();
+            cp_async_wait<1>();                                        // arrival 0 landed
+            __syncthreads();
+        }
+        for (uint32_t k = 0; k < kn; ++k) {
+            const uint32_t now = tick0 + k0 + k;
+            const int32_t inc = s_arr[k];
+            const float *row_inc, *col_inc;
+            uint32_t col_stride;
+            if (g.matrix_mode == 1) {
+                // arrival k's row and column are in the ring (made visible by the last barrier)
+                if (k + 2 < kn) prefetch(k + 2, s_arr[k + 2]);
+                cp_async_commit();
+                row_inc = s_mat + (size_t)(k % kRing) * 2 * P; col_inc = row_inc + P; col_stride = 1;
+            } else if (g.matrix_mode == 0) {
+                row_inc = s_mat + (size_t)inc * P; col_inc = s_mat + inc; col_stride = P;
+            } else {
+                row_inc = Pm + (size_t)inc * P; col_inc = Pm + inc; col_stride = P;
             }
-        } else if (tid == (uint32_t)(best & 0xffffffffu)) {
-            const uint32_t life = __ldg(&g.arr_life[k]);
-            for (uint32_t t = 0; t < c; ++t)              // the what-if sums become the cached ones
-                my_part[t] = __fadd_rn(my_part[t], Pm[(size_t)my_ids[t] * g.P + inc]);
-            my_part[c] = mu_inc;
-            my_ids[c] = inc;
-            const uint32_t e = life ? now + life : 0u;
-            my_exp[c] = e;
-            if (e && e < next_exp) next_exp = e;
-            ++c;
-            g.gpu_out[k] = (int32_t)tid;
-            if (g.mean_out) g.mean_out[k] = mean;
-            if (g.mu_arr_out) g.mu_arr_out[k] = mu_inc;
+            unsigned long long key = kNoGpu;
+            float mean = 0.0f, mu_inc = 0.0f;
+            if (owner) {
+                if (next_exp <= now) {                                 // departures, order kept
+                    unsigned long long keep = 0;
+                    for (uint32_t s = 0; s < c; ++s) {
+                        const uint32_t e = EX(s);
+                        if (!(e != 0 && e <= now)) keep |= 1ull << s;
+                    }
+                    uint32_t w = 0;
+                    next_exp = 0xffffffffu;
+                    for (uint32_t s = 0; s < c; ++s) {
+                        if (!((keep >> s) & 1ull)) continue;
+                        const uint32_t e = EX(s);
+                        ID(w) = ID(s); EX(w) = e;
+                        if (e && e < next_exp) next_exp = e;
+                        if (g.pair_cache) {                              // survivors' terms, same order
+                            uint32_t v = 0;
+                            for (uint32_t u = 0; u < c; ++u)
+                                if ((keep >> u) & 1ull) { PT(w, v) = PT(s, u); ++v; }
+                        }
+                        ++w;
+                    }
+                    for (uint32_t s = w; s < c; ++s) { ID(s) = -1; EX(s) = 0; }
+                    c = w;
+                    recompute_partials(c);
+                }
+                if (c < R) {                                           // what-if: residents + the arrival
+                    float tot = 0.0f;
+                    if constexpr (kSlots > 0) {
+                        float to_inc[kSlots], from_inc[kSlots], part[kSlots];
+#pragma unroll
+                        for (int t = 0; t < kSlots; ++t) {
+                            if ((uint32_t)t < c) {
+                                const int32_t id = ID(t);
+                                part[t] = PA(t);
+                                to_inc[t] = col_inc[(size_t)id * col_stride];   // P[id][inc]
+                                from_inc[t] = row_inc[id];                       // P[inc][id]
+                            }
+                        }
+#pragma unroll
+                        for (int t = 0; t < kSlots; ++t) {
+                            if ((uint32_t)t < c) {
+                                tot = __fadd_rn(tot, __fadd_rn(part[t], to_inc[t]));
+                                mu_inc = __fadd_rn(mu_inc, from_inc[t]);
+                            }
+                        }
+                    } else {
+                        for (uint32_t t = 0; t < c; ++t) {
+                            const int32_t id = ID(t);
+                            tot = __fadd_rn(tot, __fadd_rn(PA(t), col_inc[(size_t)id * col_stride]));
+                            mu_inc = __fadd_rn(mu_inc, row_inc[id]);
+                        }
+                    }
+                    tot = __fadd_rn(tot, mu_inc);
+                    mean = __fdiv_rn(tot, (float)(c + 1));
+                    if (mean < g.lambda)                               // Algorithm 2 line 7
+                        key = ((unsigned long long)__float_as_uint(mean) << 32) | tid;
+                }
+            }
+            // argmin over GPUs, lowest index on equal means (mean >= 0, so its bits order as integers)
+            const uint32_t hi = (uint32_t)(key >> 32);
+            const uint32_t best_hi = __reduce_min_sync(0xffffffffu, hi);
+            const uint32_t best_lo = __reduce_min_sync(0xffffffffu, hi == best_hi ? (uint32_t)key : 0xffffffffu);
+            if (lane == 0) s_key[k & 1][wid] = ((unsigned long long)best_hi << 32) | best_lo;
+            if (g.matrix_mode == 1) cp_async_wait<1>();                // this thread's share of arrival k+1 landed
+            __syncthreads();
+            unsigned long long best = s_key[k & 1][0];
+            for (uint32_t w = 1; w < nwarps; ++w) {
+                const unsigned long long o = s_key[k & 1][w];
+                best = o < best ? o : best;
+            }
+            if (best == kNoGpu) {
+                if (tid == 0) {
+                    g.gpu_out[k0 + k] = -1;
+                    if (g.mean_out) g.mean_out[k0 + k] = 0.0f;
+                    if (g.mu_arr_out) g.mu_arr_out[k0 + k] = 0.0f;
+                }
+            } else if (tid == (uint32_t)(best & 0xffffffffu)) {
+                const uint32_t life = (uint32_t)s_arr[kArrChunk + k];
+                for (uint32_t t = 0; t < c; ++t) {                     // the what-if sums become the cached ones
+                    const float to = col_inc[(size_t)ID(t) * col_stride];
+                    PA(t) = __fadd_rn(PA(t), to);
+                    if (g.pair_cache) { PT(t, c) = to; PT(c, t) = row_inc[ID(t)]; }
+                }
+                if (g.pair_cache) PT(c, c) = 0.0f;
+                PA(c) = mu_inc;
+                ID(c) = inc;
+                const uint32_t e = life ? now + life : 0u;
+                EX(c) = e;
+                if (e && e < next_exp) next_exp = e;
+                ++c;
+                g.gpu_out[k0 + k] = (int32_t)tid;
+                if (g.mean_out) g.mean_out[k0 + k] = mean;
+                if (g.mu_arr_out) g.mu_arr_out[k0 + k] = mu_inc;
+            }
         }
+        if (g.matrix_mode == 1) cp_async_wait<0>();
     }
     if (owner) g.count[tid] = c;
     __syncthreads();
-    for (uint32_t i = tid; i < GR; i += blockDim.x) { g.ids[i] = s_ids[i]; g.expiry[i] = s_exp[i]; }
+    for (uint32_t i = tid; i < GR; i += blockDim.x) {
+        const uint32_t gpu = i / R, slot = i % R;
+        g.ids[i] = s_ids[slot * G + gpu];
+        g.expiry[i] = s_exp[slot * G + gpu];
+    }
     if (tid == 0) *g.tick = tick0 + g.n;
 }
 
@@ -209,14 +317,23 @@ extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_
     a.ids = state->ids; a.expiry = state->expiry; a.count = state->count; a.tick = state->tick;
     a.arr_id = arr_id; a.arr_life = arr_life; a.n = n; a.lambda = opts->lambda;
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
-    const size_t state_bytes = (size_t)a.G * a.R * 12;
-    const size_t mat_bytes = (size_t)P * P * sizeof(float);
-    a.matrix_in_smem = state_bytes + mat_bytes <= 160 * 1024;
-    const size_t smem = state_bytes + (a.matrix_in_smem ? mat_bytes : 0);
+    size_t state_bytes = (size_t)a.G * a.R * 12 + 2 * kArrChunk * sizeof(int32_t);
+    const size_t pair_bytes = (size_t)a.G * a.R * a.R * sizeof(float);
+    a.pair_cache = pair_bytes <= 64 * 1024;
+    if (a.pair_cache) state_bytes += pair_bytes;
+    const size_t mat_bytes = (size_t)P * P * sizeof(float), ring_bytes = (size_t)kRing * 2 * P * sizeof(float);
+    const size_t budget = 200 * 1024;
+    size_t smem = state_bytes;
+    if (state_bytes + mat_bytes <= budget) { a.matrix_mode = 0; smem += mat_bytes; }
+    else if (state_bytes + ring_bytes <= budget) { a.matrix_mode = 1; smem += ring_bytes; }
+    else a.matrix_mode = 2;
+    uint32_t threads = ((a.G + 31) / 32) * 32;
+    if (a.matrix_mode == 1 && threads < 128) threads = 128;          // more lanes to issue the prefetch
+    auto kern = a.R <= 4 ? place_kernel<4> : a.R <= 8 ? place_kernel<8> : a.R <= 16 ? place_kernel<16>
+                                                                                   : place_kernel<0>;
     if (smem > 48 * 1024)
-        ROOMIE_CUDA_OK(cudaFuncSetAttribute(place_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const uint32_t threads = ((a.G + 31) / 32) * 32;
-    place_kernel<<<1, threads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+        ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<1, threads, smem, static_cast<cudaStream_t>(stream)>>>(a);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;

@@ -38,5 +38,5 @@ def test_host_side_argument_checks():
     class Spec(ctypes.Structure):
         _fields_ = [(n, ctypes.c_uint32) for n in "abcde"]
     dll.roomie_share_table_floats.restype = ctypes.c_size_t
-    assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 65536, 164 * 1024, 2048, 32))) == 2 * 65 * 65
+    assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 65536, 164 * 1024, 2048, 32))) == 2 * 64 + 1
     assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 1 << 18, 164 * 1024, 2048, 32))) == 0   # RANGE

@@ -328,6 +328,9 @@ def test_placement_edge_cases(rm, oracle):
         (1, 1, [-1], [0], [0] * 4, [1] * 4, 0.5),
         (1, 1, [-1], [0], [0] * 4, [2] * 4, 0.5),
         (33, 3, [-1] * 99, [0] * 33, list(range(3)) * 40, [5] * 120, 0.3),
+        (3, 12, [-1] * 36, [0] * 3, list(range(3)) * 30, [7] * 90, 2.6),      # 9..16 slots: unrolled by 16
+        (5, 20, [-1] * 100, [0] * 5, list(range(3)) * 60, [50] * 180, 4.1),   # > 16 slots: plain loops
+        (40, 24, [-1] * 960, [0] * 40, list(range(3)) * 400, [300] * 1200, 5.0),  # resident terms not cached
     ]
     for G, R, ids, count, aid, life, lam in cases:
         st = rm.ClusterState(G, R, ids, [0] * (G * R), count, 7)
@@ -343,4 +346,12 @@ def test_placement_edge_cases(rm, oracle):
     st = rm.ClusterState(cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0)
     gpu = rm.place(big, st, cl.arr_id, cl.arr_life, 0.5)[0].cpu().numpy()
     want = oracle.place(big, cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0, cl.arr_id, cl.arr_life, 0.5)
+    assert np.array_equal(gpu, want.gpu)
+    # matrix too large even for the row/column ring -> plain global loads
+    P = 6600
+    huge = rng.random((P, P), dtype=np.float32) * np.float32(0.3)
+    cl = rs.make_cluster(2, num_profiles=P, num_arrivals=300)
+    st = rm.ClusterState(cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0)
+    gpu = rm.place(huge, st, cl.arr_id, cl.arr_life, 0.5)[0].cpu().numpy()
+    want = oracle.place(huge, cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0, cl.arr_id, cl.arr_life, 0.5)
     assert np.array_equal(gpu, want.gpu)
