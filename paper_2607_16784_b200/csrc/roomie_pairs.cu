@@ -19,7 +19,6 @@ namespace roomie {
 constexpr int kTileThreads = 128;
 constexpr int kItems = 16;                              // path steps per thread
 constexpr int kTileItems = kTileThreads * kItems;       // path steps per tile
-constexpr int kFinalThreads = 128;
 
 struct PairSet {                  // which pairs a launch covers
     uint64_t pair_begin;          // first triangular pair index (explicit == 0)
@@ -210,16 +209,22 @@ struct TileArgs {
     PhiCap cap;
 };
 
-// Shared-memory layout of one tile.  Records are padded by one slot after every 8 so that the
-// lanes of a warp, whose positions on the merge path are about 8 records apart, fall into
-// different bank groups; the search keys (end ticks, re-based) live in their own array with
-// one pad word per 32 so that the binary-search probes of a warp do not collide either.
+// Shared-memory layout of one tile.  The tile's A records sit at unified indices 0, 1, 2, ... and
+// its B records at kTileLoad-1, kTileLoad-2, ... (the two runs never meet: together they hold at
+// most kTileLoad records).  Records are padded by one slot after every 8 so that the lanes of a
+// warp, whose positions on the merge path are about 8 records apart, fall into different bank
+// groups; the search keys (end ticks) live in their own array with one pad word per 32 so that
+// the binary-search probes of a warp do not collide either.  Both paddings are linear in the
+// staging loop's trip count, so staging addresses are base + immediate.
+// Staged A records carry the *slack* Phi|guards - phi_a in place of phi_a; B records keep phi_b:
+// Eq. 2 for a pairing is then two subtractions and a test of the guard bits.
 __device__ __forceinline__ uint32_t rec_slot(uint32_t i) { return i + (i >> 3); }
 __device__ __forceinline__ uint32_t key_slot(uint32_t i) { return i + (i >> 5); }
 constexpr int kTileLoad = kTileItems + 2;                               // one look-ahead record per side
 constexpr int kRecSlots = kTileLoad + (kTileLoad >> 3) + 2;
 constexpr int kKeySlots = kTileLoad + (kTileLoad >> 5) + 2;
 constexpr int kStageBatch = 6;                                           // global loads in flight per thread
+constexpr int kStageRounds = (kTileLoad + kTileThreads * kStageBatch - 1) / (kTileThreads * kStageBatch);
 
 template <bool kWithV>
 __device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned long long V, uint32_t ties,
@@ -248,6 +253,60 @@ __device__ __forceinline__ float small_int_to_float(uint32_t v) {
     return __uint_as_float(0x4B000000u | v) - 8388608.0f;
 }
 
+// one side of the staging: records src[0..n) -> unified indices first, first+step, ...
+// (step = +1 for A, -1 for B); kSlack: store cap - phi instead of phi
+template <bool kSlack, int kDir>
+__device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32_t n, uint32_t base_tick, PhiCap cap,
+                                           uint4* s_rec, int32_t* s_key) {
+    // thread t handles records t, t + 128, ...; 128 is a multiple of 8 and 32, so both paddings
+    // advance by a constant per trip
+    const uint32_t i0 = kDir > 0 ? threadIdx.x : (uint32_t)(kTileLoad - 1) - threadIdx.x;
+    uint4* rp = s_rec + rec_slot(i0);
+    int32_t* kp = s_key + key_slot(i0);
+    constexpr int kRecStep = kDir * (kTileThreads + kTileThreads / 8);
+    constexpr int kKeyStep = kDir * (kTileThreads + kTileThreads / 32);
+#pragma unroll
+    for (int round = 0; round < kStageRounds; ++round) {
+        const uint32_t r0 = threadIdx.x + round * kStageBatch * kTileThreads;
+        if (r0 >= n) break;
+        uint4 r[kStageBatch];
+#pragma unroll
+        for (int j = 0; j < kStageBatch; ++j)
+            if (r0 + j * kTileThreads < n) r[j] = __ldg(src + r0 + j * kTileThreads);
+#pragma unroll
+        for (int j = 0; j < kStageBatch; ++j) {
+            if (r0 + j * kTileThreads < n) {
+                r[j].x -= base_tick; r[j].y -= base_tick;
+                if (kSlack) { r[j].z = cap.lo - r[j].z; r[j].w = cap.hi - r[j].w; }
+                rp[(round * kStageBatch + j) * kRecStep] = r[j];
+                kp[(round * kStageBatch + j) * kKeyStep] = (int32_t)r[j].y;
+            }
+        }
+    }
+}
+
+// one step of the walk for the pairing (ra, rb).  A step that is not live (ragged tail of a walk)
+// touches nothing: the registers may then hold a record from beyond the staged range.
+#define ROOMIE_WALK_STEP(live)                                                                         \
+    if (live) {                                                                                        \
+        const int32_t Ea = (int32_t)ra.y, Eb = (int32_t)rb.y;                                          \
+        const int32_t ov = min(Ea, Eb) - max((int32_t)ra.x, (int32_t)rb.x);                            \
+        const bool hit = (ov > 0) && phi_exceeds(ra.z, ra.w, rb.z, rb.w);                              \
+        const float tw = (hit ? (float)ov : 0.0f) * s_inv[wsum_b - wslack_a];   /* overlap/(o_i+o_j) */ \
+        di = fmaf(tw, fa, di);                                                                         \
+        dj = fmaf(tw, fb, dj);                                                                         \
+        if (kWithV) V += hit ? (unsigned long long)(uint32_t)ov : 0ull;                                \
+        ties += (Ea == Eb) ? 1u : 0u;                                                                  \
+        if (Ea <= Eb) {                                                                                \
+            ++x; ra = s_rec[rec_slot(x)];                                                              \
+            wslack_a = ra.z >> kWarpShift; fa = small_int_to_float(wconst - wslack_a);                 \
+        } else {                                                                                       \
+            --ib; rb = s_rec[rec_slot(ib)];                                                            \
+            const uint32_t wb = rb.z >> kWarpShift;                                                    \
+            wsum_b = wb + wconst; fb = small_int_to_float(wb);                                         \
+        }                                                                                              \
+    }
+
 template <bool kWithV>
 __global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArgs g) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -260,31 +319,15 @@ __global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArg
 
     for (uint32_t i = threadIdx.x; i < g.n_inv; i += kTileThreads) s_inv[i] = __ldg(&g.inv_table[i]);
     const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
+    // warps field of a staged A record holds (W + guard) - warps_a
+    const uint32_t wconst = g.cap.lo >> kWarpShift;
 
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
         const TileDesc d = g.tiles[t];
         const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
-        const uint32_t n_load = loadA + loadB;
         __syncthreads();                                   // previous tile fully consumed
-        // stage the tile: A records first, then B; ticks re-based to the alignment's start
-        for (uint32_t i0 = threadIdx.x; i0 < n_load; i0 += kTileThreads * kStageBatch) {
-            uint4 r[kStageBatch];
-#pragma unroll
-            for (int j = 0; j < kStageBatch; ++j) {
-                const uint32_t i = i0 + j * kTileThreads;
-                if (i < n_load) r[j] = __ldg(i < loadA ? &g.records[d.recA + i] : &g.records[d.recB + (i - loadA)]);
-            }
-#pragma unroll
-            for (int j = 0; j < kStageBatch; ++j) {
-                const uint32_t i = i0 + j * kTileThreads;
-                if (i < n_load) {
-                    const uint32_t base = i < loadA ? d.baseA : d.baseB;
-                    r[j].x -= base; r[j].y -= base;
-                    s_rec[rec_slot(i)] = r[j];
-                    s_key[key_slot(i)] = (int32_t)r[j].y;
-                }
-            }
-        }
+        stage_side<true, +1>(g.records + d.recA, loadA, d.baseA, g.cap, s_rec, s_key);
+        stage_side<false, -1>(g.records + d.recB, loadB, d.baseB, g.cap, s_rec, s_key);
         __syncthreads();
         const uint32_t len = d.cntA + d.cntB;
         const uint32_t diag = threadIdx.x * kItems;
@@ -292,43 +335,31 @@ __global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArg
         unsigned long long V = 0;
         uint32_t ties = 0;
         if (diag < len) {
-            // this thread's start point on the tile's merge path (A first on equal end times)
+            // this thread's start point on the tile's merge path (A first on equal end times):
+            // B record y sits at unified index kTileLoad - 1 - y
             uint32_t lo = diag > d.cntB ? diag - d.cntB : 0u, hi = diag < d.cntA ? diag : d.cntA;
+            const uint32_t btop = (uint32_t)kTileLoad - diag;              // index of B[diag - 1 - mid] is btop + mid
             while (lo < hi) {
                 const uint32_t mid = (lo + hi) >> 1;
-                if (s_key[key_slot(mid)] <= s_key[key_slot(loadA + diag - 1 - mid)]) lo = mid + 1; else hi = mid;
+                if (s_key[key_slot(mid)] <= s_key[key_slot(btop + mid)]) lo = mid + 1; else hi = mid;
             }
-            uint32_t x = lo, y = loadA + diag - lo;                   // unified record indices
-            const uint32_t steps = (len - diag < (uint32_t)kItems) ? len - diag : (uint32_t)kItems;
-            uint4 ra = s_rec[rec_slot(x)], rb = s_rec[rec_slot(y)];
-            uint32_t slack_lo = g.cap.lo - ra.z, slack_hi = g.cap.hi - ra.w;
-            uint32_t wa = ra.z >> kWarpShift, wb = rb.z >> kWarpShift;
-            float fa = small_int_to_float(wa), fb = small_int_to_float(wb);
+            uint32_t x = lo, ib = (uint32_t)(kTileLoad - 1) - (diag - lo);
+            uint4 ra = s_rec[rec_slot(x)], rb = s_rec[rec_slot(ib)];
+            uint32_t wslack_a = ra.z >> kWarpShift, wsum_b = (rb.z >> kWarpShift) + wconst;
+            float fa = small_int_to_float(wconst - wslack_a), fb = small_int_to_float(rb.z >> kWarpShift);
+            if (len - diag >= (uint32_t)kItems) {
 #pragma unroll
-            for (int s = 0; s < kItems; ++s) {
-                if ((uint32_t)s < steps) {
-                    const int32_t Ea = (int32_t)ra.y, Eb = (int32_t)rb.y;
-                    const int32_t ov = min(Ea, Eb) - max((int32_t)ra.x, (int32_t)rb.x);
-                    const bool hit = (ov > 0) && phi_exceeds(slack_lo, slack_hi, rb.z, rb.w);
-                    const float tw = (hit ? (float)ov : 0.0f) * s_inv[wa + wb];   // overlap / (o_i + o_j)
-                    di = fmaf(tw, fa, di);
-                    dj = fmaf(tw, fb, dj);
-                    if (kWithV) V += hit ? (unsigned long long)(uint32_t)ov : 0ull;
-                    ties += (Ea == Eb) ? 1u : 0u;
-                    if (Ea <= Eb) {
-                        ++x; ra = s_rec[rec_slot(x)];
-                        slack_lo = g.cap.lo - ra.z; slack_hi = g.cap.hi - ra.w;
-                        wa = ra.z >> kWarpShift; fa = small_int_to_float(wa);
-                    } else {
-                        ++y; rb = s_rec[rec_slot(y)];
-                        wb = rb.z >> kWarpShift; fb = small_int_to_float(wb);
-                    }
-                }
+                for (int s = 0; s < kItems; ++s) ROOMIE_WALK_STEP(true)
+            } else {
+                const uint32_t steps = len - diag;
+#pragma unroll
+                for (int s = 0; s < kItems; ++s) ROOMIE_WALK_STEP((uint32_t)s < steps)
             }
         }
         block_reduce_store<kWithV>(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
     }
 }
+#undef ROOMIE_WALK_STEP
 
 // ---------------------------------------------------------------------------------------
 // LOCKSTEP tiles (Algorithm 1 as printed): pairing t of the walk is (s_i + t, s_j + t)
@@ -373,43 +404,59 @@ struct FinalArgs {
     roomie_pair_detail detail;    // capacity 0 = none
 };
 
-// k-th smallest of v[0..n) by rank counting (ties ordered by index); every thread returns it
-__device__ float select_rank(const float* v, uint32_t n, uint32_t k, float* s_pick) {
-    for (uint32_t e = threadIdx.x; e < n; e += kFinalThreads) {
+// k-th smallest of v[0..n) by rank counting (ties ordered by index); one warp, every lane returns it
+__device__ float select_rank(const float* v, uint32_t n, uint32_t k, int lane) {
+    float pick = 0.0f;
+    bool mine = false;
+    for (uint32_t e = lane; e < n; e += 32) {
         const float x = v[e];
         uint32_t rank = 0;
         for (uint32_t j = 0; j < n; ++j) {
             const float y = v[j];
             rank += (y < x) || (y == x && j < e);
         }
-        if (rank == k) *s_pick = x;
+        if (rank == k) { pick = x; mine = true; }
     }
-    __syncthreads();
-    const float r = *s_pick;
-    __syncthreads();
-    return r;
+    const uint32_t who = __ballot_sync(0xffffffffu, mine);        // exactly one lane holds rank k
+    return __shfl_sync(0xffffffffu, pick, __ffs(who) - 1);
 }
 
-__global__ void __launch_bounds__(kFinalThreads) finalize_kernel(FinalArgs g) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float* v_i = reinterpret_cast<float*>(smem_raw);
-    float* v_j = v_i + g.slots;
-    __shared__ uint32_t s_warp[kFinalThreads / 32];
-    __shared__ float s_pick;
-    __shared__ unsigned long long s_ev[kFinalThreads / 32];
+// P[a][b], P[b][a] from the two medians (gamma = max(q_i/q_j, 1), Eq. 4 with M = {i, j})
+__device__ __forceinline__ void store_pair(const FinalArgs& g, uint32_t a, uint32_t b, uint32_t qa, uint32_t qb,
+                                           float med_i, float med_j) {
+    const unsigned long long Ta = g.lib.T[a], Tb = g.lib.T[b];
+    const float fa = (float)qa, fb = (float)qb;
+    const float g_ab = fmaxf(__fdiv_rn(fa, fb), 1.0f), g_ba = fmaxf(__fdiv_rn(fb, fa), 1.0f);
+    const float p_ab = Ta ? __fdiv_rn(g_ab * med_i, (float)Ta) : 0.0f;
+    const float p_ba = Tb ? __fdiv_rn(g_ba * med_j, (float)Tb) : 0.0f;
+    if (g.ps.explicit_pair) {
+        g.P_out[0] = p_ab; g.P_out[1] = p_ba;
+    } else {
+        g.P_out[(size_t)a * g.lib.P + b] = p_ab;
+        if (a != b) g.P_out[(size_t)b * g.lib.P + a] = p_ba;
+    }
+}
 
-    const uint32_t local = blockIdx.x;
+// one warp per pair: ordered sum of the tile partials of every alignment, ordered compaction of
+// the kept alignments, medians by rank counting
+constexpr int kFinalWarps = 8;
+__global__ void __launch_bounds__(kFinalWarps * 32) finalize_kernel(FinalArgs g) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const uint32_t local = blockIdx.x * (blockDim.x >> 5) + wid;
+    if (local >= g.ps.n_pairs) return;                       // whole warp leaves together
+    float* v_i = reinterpret_cast<float*>(smem_raw) + (size_t)wid * 2 * g.slots;
+    float* v_j = v_i + g.slots;
     uint32_t a, b;
     pair_of(g.ps, g.lib.P, local, a, b);
     const uint32_t qa = g.lib.offsets[a + 1] - g.lib.offsets[a], qb = g.lib.offsets[b + 1] - g.lib.offsets[b];
     const uint32_t gb = grid_count(qb, g.n_align);
     const WalkInfo* walks = g.walks + (size_t)local * g.slots;
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 
-    uint32_t kept_before = 0;
+    uint32_t n = 0;
     unsigned long long evals = 0;
-    for (uint32_t c0 = 0; c0 < g.slots; c0 += kFinalThreads) {
-        const uint32_t c = c0 + threadIdx.x;
+    for (uint32_t c0 = 0; c0 < g.slots; c0 += 32) {
+        const uint32_t c = c0 + lane;
         bool valid = false;
         float di = 0.0f, dj = 0.0f;
         unsigned long long V = 0;
@@ -427,14 +474,8 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(FinalArgs g) {
                 evals += ev;
             }
         }
-        // ordered compaction of the kept alignments
         const uint32_t ballot = __ballot_sync(0xffffffffu, valid);
-        if (lane == 0) s_warp[wid] = __popc(ballot);
-        __syncthreads();
-        uint32_t pos = kept_before + __popc(ballot & ((1u << lane) - 1u));
-        uint32_t chunk = 0;
-#pragma unroll
-        for (int w = 0; w < kFinalThreads / 32; ++w) { if (w < wid) pos += s_warp[w]; chunk += s_warp[w]; }
+        const uint32_t pos = n + __popc(ballot & ((1u << lane) - 1u));
         if (valid) {
             v_i[pos] = di; v_j[pos] = dj;
             if (pos < g.detail.capacity) {
@@ -447,43 +488,51 @@ __global__ void __launch_bounds__(kFinalThreads) finalize_kernel(FinalArgs g) {
                 if (g.detail.evals) g.detail.evals[pos] = ev;
             }
         }
-        kept_before += chunk;
-        __syncthreads();
+        n += __popc(ballot);
     }
-    const uint32_t n = kept_before;
+    __syncwarp();
     float med_i = 0.0f, med_j = 0.0f;
     if (n > 0) {
         const uint32_t k1 = (n - 1) / 2, k2 = n / 2;
-        const float i1 = select_rank(v_i, n, k1, &s_pick);
-        const float i2 = (k2 == k1) ? i1 : select_rank(v_i, n, k2, &s_pick);
-        const float j1 = select_rank(v_j, n, k1, &s_pick);
-        const float j2 = (k2 == k1) ? j1 : select_rank(v_j, n, k2, &s_pick);
+        const float i1 = select_rank(v_i, n, k1, lane);
+        const float i2 = (k2 == k1) ? i1 : select_rank(v_i, n, k2, lane);
+        const float j1 = select_rank(v_j, n, k1, lane);
+        const float j2 = (k2 == k1) ? j1 : select_rank(v_j, n, k2, lane);
         med_i = 0.5f * (i1 + i2);
         med_j = 0.5f * (j1 + j2);
     }
 #pragma unroll
     for (int s = 16; s > 0; s >>= 1) evals += __shfl_xor_sync(0xffffffffu, evals, s);
-    if (lane == 0) s_ev[wid] = evals;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned long long Ta = g.lib.T[a], Tb = g.lib.T[b];
-        const float fa = (float)qa, fb = (float)qb;
-        const float g_ab = fmaxf(__fdiv_rn(fa, fb), 1.0f), g_ba = fmaxf(__fdiv_rn(fb, fa), 1.0f);
-        const float p_ab = Ta ? __fdiv_rn(g_ab * med_i, (float)Ta) : 0.0f;
-        const float p_ba = Tb ? __fdiv_rn(g_ba * med_j, (float)Tb) : 0.0f;
-        if (g.ps.explicit_pair) {
-            g.P_out[0] = p_ab; g.P_out[1] = p_ba;
-        } else {
-            g.P_out[(size_t)a * g.lib.P + b] = p_ab;
-            if (a != b) g.P_out[(size_t)b * g.lib.P + a] = p_ba;
-        }
+    if (lane == 0) {
+        store_pair(g, a, b, qa, qb, med_i, med_j);
         if (g.detail.n_kept) *g.detail.n_kept = n;
-        if (g.evals_out) {
-            unsigned long long tot = 0;
-            for (int w = 0; w < kFinalThreads / 32; ++w) tot += s_ev[w];
-            atomicAdd(g.evals_out, tot);
-        }
+        if (g.evals_out && evals) atomicAdd(g.evals_out, evals);
     }
+}
+
+// one alignment per pair and no per-alignment outputs (the base setting): one thread per pair
+__global__ void __launch_bounds__(256) finalize_single_kernel(FinalArgs g) {
+    const uint32_t local = blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long evals = 0;
+    if (local < g.ps.n_pairs) {
+        uint32_t a, b;
+        pair_of(g.ps, g.lib.P, local, a, b);
+        const uint32_t qa = g.lib.offsets[a + 1] - g.lib.offsets[a], qb = g.lib.offsets[b + 1] - g.lib.offsets[b];
+        const WalkInfo wi = g.walks[local];
+        float di = 0.0f, dj = 0.0f;
+        if (wi.valid) {
+            uint32_t ties = 0;
+            for (uint32_t k = 0; k < wi.n_tiles; ++k) {
+                const TilePartial p = g.partials[wi.tile_base + k];
+                di += p.di; dj += p.dj; ties += p.ties;
+            }
+            evals = wi.length - ties;
+        }
+        store_pair(g, a, b, qa, qb, 0.5f * (di + di), 0.5f * (dj + dj));   // median of one value, same arithmetic
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) evals += __shfl_xor_sync(0xffffffffu, evals, s);
+    if ((threadIdx.x & 31) == 0 && g.evals_out && evals) atomicAdd(g.evals_out, evals);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -622,7 +671,16 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
     fa.lib = lv; fa.ps = ps; fa.slots = slots; fa.n_align = o->n_align; fa.walks = walks; fa.partials = partials;
     fa.P_out = P_out; fa.evals_out = reinterpret_cast<unsigned long long*>(evals_out);
     if (detail) fa.detail = *detail; else { roomie_pair_detail z = {}; fa.detail = z; }
-    finalize_kernel<<<ps.n_pairs, kFinalThreads, (size_t)slots * 2 * sizeof(float), st>>>(fa);
+    if (slots == 1 && !detail) {
+        finalize_single_kernel<<<(ps.n_pairs + 255) / 256, 256, 0, st>>>(fa);
+    } else {
+        uint32_t wpb = (uint32_t)((96 * 1024) / ((size_t)slots * 2 * sizeof(float)));   // warps (= pairs) per CTA
+        wpb = wpb < 1 ? 1 : (wpb > kFinalWarps ? kFinalWarps : wpb);
+        const size_t fsmem = (size_t)wpb * slots * 2 * sizeof(float);
+        if (fsmem > 48 * 1024)
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsmem));
+        finalize_kernel<<<(ps.n_pairs + wpb - 1) / wpb, wpb * 32, fsmem, st>>>(fa);
+    }
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;

@@ -67,6 +67,7 @@ struct PlaceArgs {
     float* mu_arr_out;
     int matrix_mode;        // 0: whole matrix in shared memory, 1: row/column ring, 2: global loads
     int pair_cache;         // 1: resident-resident terms cached in shared memory ([R][R][G] floats)
+    uint32_t gpus_per_warp; // fast kernel: GPUs owned by each warp
 };
 
 constexpr unsigned long long kNoGpu = ~0ull;
@@ -285,6 +286,229 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
     if (tid == 0) *g.tick = tick0 + g.n;
 }
 
+// ---------------------------------------------------------------------------------------
+// K5, fast variant for up to 8 slots per GPU.  On top of the scheme above it keeps the matrix
+// off the critical path entirely, whatever its size:
+//   - every resident sits in a fixed *physical* slot; the arrival order of a GPU's residents is a
+//     packed nibble list in a register, so a departure moves no shared-memory data and copies in
+//     flight never have to follow a resident;
+//   - at arrival j each thread issues cp.async for the 2 matrix elements per resident that
+//     arrival j+3 will need, into a 4-deep ring indexed by physical slot;
+//   - a resident younger than 3 arrivals is not covered by the ring (it was placed after the
+//     fetch was issued); its terms depend only on the arrival stream (P[arr_{j-d}][arr_j] and the
+//     transpose, d = 1..3) and are fetched by six designated threads on the same schedule.
+// The critical path per arrival is shared-memory reads, 2c+2 float adds, one division, two
+// redux steps and one barrier.
+// ---------------------------------------------------------------------------------------
+constexpr int kAhead = 3;                     // arrivals fetched ahead
+constexpr int kYoungRing = 8;                 // ring depth of the arrival-to-arrival terms
+constexpr int kYoungInit = -(1 << 30);        // birth index of initial residents
+
+__device__ __forceinline__ void cp_async_4_s(uint32_t smem_addr, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(smem_addr), "l"(gmem_src) : "memory");
+}
+
+__global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
+    // one float/int array; every region is addressed by a 32-bit word index
+    extern __shared__ __align__(16) float sm[];
+    int32_t* smi = reinterpret_cast<int32_t*>(sm);
+    uint32_t* smu = reinterpret_cast<uint32_t*>(sm);
+    const uint32_t G = g.G, R = g.R, P = g.P, GR = G * R;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = blockDim.x >> 5;
+    // GPUs are spread over the warps (gpw per warp, low lanes) so that the serial sections of an
+    // arrival - a departure on one GPU, the winner's update on another - run in different warps;
+    // the last warp owns no GPU and fetches the arrival-to-arrival terms
+    const uint32_t gpw = g.gpus_per_warp;
+    const uint32_t gpu = wid * gpw + lane;
+    const bool helper = wid == nwarps - 1;
+    // word offsets of the regions; per-GPU arrays are [slot][gpu]
+    const uint32_t oID = gpu, oEX = GR + gpu, oPA = 2 * GR + gpu, oBI = 3 * GR + gpu;
+    const uint32_t oPT = 4 * GR + gpu;                    // [slot][slot][gpu]
+    const uint32_t oRING = 4 * GR + GR * R + gpu;         // [4][2][slot][gpu]
+    const uint32_t oYOUNG = 4 * GR + GR * R + 8 * GR;     // [kYoungRing][kAhead][2]
+    const uint32_t oARR = oYOUNG + kYoungRing * kAhead * 2;   // ids [kArrChunk + 2 kAhead], then lifetimes [kArrChunk]
+    const uint32_t oLIFE = oARR + kArrChunk + 2 * kAhead;
+    const uint32_t oOUT = oLIFE + kArrChunk;              // decisions of the chunk: gpu, mean, mu_arr [3][kArrChunk]
+    const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(sm);
+    __shared__ unsigned long long s_key[2][32];
+
+    const float* __restrict__ Pm = g.Pm;
+    const bool owner = !helper && lane < gpw && gpu < G;
+
+    // initial state: residents occupy physical slots 0..c-1 in arrival order
+    uint32_t c = 0, ord = 0, free_mask = (1u << R) - 1u, next_exp = 0xffffffffu;
+    if (owner) {
+        c = min(g.count[gpu], R);
+        for (uint32_t p = 0; p < R; ++p) {
+            smi[oID + p * G] = p < c ? g.ids[gpu * R + p] : -1;
+            smu[oEX + p * G] = p < c ? g.expiry[gpu * R + p] : 0u;
+            smi[oBI + p * G] = kYoungInit;
+        }
+        for (uint32_t p = 0; p < c; ++p) {
+            ord |= p << (4 * p);
+            free_mask &= ~(1u << p);
+            const uint32_t e = smu[oEX + p * G];
+            if (e && e < next_exp) next_exp = e;
+            for (uint32_t q = 0; q < c; ++q)
+                sm[oPT + (p * R + q) * G] = __ldg(&Pm[(size_t)smi[oID + p * G] * P + smi[oID + q * G]]);
+        }
+        for (uint32_t p = 0; p < c; ++p) {
+            float s = 0.0f;
+            for (uint32_t q = 0; q < c; ++q)
+                if (q != p) s = __fadd_rn(s, sm[oPT + (p * R + q) * G]);
+            sm[oPA + p * G] = s;
+        }
+    }
+    const uint32_t tick0 = *g.tick;
+
+    // fetch what arrival a (s_arr index a_local, global index a_global) will need
+    auto issue = [&](uint32_t a_local, uint32_t a_global) {
+        const int32_t inc = smi[oARR + a_local];
+        const float* row = Pm + (size_t)inc * P;          // P[inc][*]
+        const float* col = Pm + inc;                      // P[*][inc]
+        const uint32_t ring = oRING + (a_global & 3u) * 2 * GR;
+        for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {      // c = 0 for threads that own no GPU
+            const uint32_t p = o & 15u;
+            const int32_t id = smi[oID + p * G];
+            cp_async_4_s(sm_base + 4u * (ring + p * G), col + (size_t)id * P);
+            cp_async_4_s(sm_base + 4u * (ring + GR + p * G), row + id);
+        }
+        if (helper && lane < 2 * kAhead) {
+            const uint32_t d = (lane >> 1) + 1, dir = lane & 1u;
+            if (a_local >= d) {
+                const int32_t old = smi[oARR + a_local - d];
+                cp_async_4_s(sm_base + 4u * (oYOUNG + ((a_global & (kYoungRing - 1)) * kAhead + (d - 1)) * 2 + dir),
+                             dir == 0 ? col + (size_t)old * P : row + old);
+            }
+        }
+    };
+    // word index of the term between the arrival kg and the resident in physical slot p:
+    // young residents read the arrival-to-arrival terms, the others the ring
+    auto term_index = [&](uint32_t kg, uint32_t p) -> uint32_t {
+        const uint32_t d1 = (uint32_t)((int32_t)(kg + 1) - smi[oBI + p * G]) - 1u;     // arrivals since placed, minus 1
+        const uint32_t iy = oYOUNG + ((kg & (kYoungRing - 1)) * kAhead + d1) * 2;
+        const uint32_t ir = oRING + (kg & 3u) * 2 * GR + p * G;
+        return d1 < (uint32_t)kAhead ? (iy | 0x80000000u) : ir;                        // top bit: young
+    };
+
+    for (uint32_t k0 = 0; k0 < g.n; k0 += kArrChunk) {
+        const uint32_t kn = min(kArrChunk, g.n - k0);
+        // stage arrival ids [k0 - kAhead, k0 + kn + kAhead) and lifetimes [k0, k0 + kn)
+        __syncthreads();
+        for (uint32_t i = tid; i < kn + 2 * kAhead; i += blockDim.x) {
+            const long long gi = (long long)k0 + i - kAhead;
+            smi[oARR + i] = (gi >= 0 && gi < (long long)g.n) ? g.arr_id[gi] : 0;
+        }
+        for (uint32_t i = tid; i < kn; i += blockDim.x) smi[oLIFE + i] = (int32_t)g.arr_life[k0 + i];
+        __syncthreads();
+        if (k0 == 0) {                                                      // prime: arrivals 0 .. kAhead-1
+            for (uint32_t a = 0; a < (uint32_t)kAhead; ++a) {
+                if (a < g.n) issue(a + kAhead, a);
+                cp_async_commit();
+            }
+            cp_async_wait<kAhead - 1>();
+            __syncthreads();
+        }
+        for (uint32_t k = 0; k < kn; ++k) {
+            const uint32_t kg = k0 + k, now = tick0 + kg, kl = k + kAhead;  // global index, tick, index into the staged ids
+            if (owner && next_exp <= now) {                                  // departures: drop from the order list
+                uint32_t w = 0, nord = 0;
+                next_exp = 0xffffffffu;
+                for (uint32_t t = 0; t < c; ++t) {
+                    const uint32_t p = (ord >> (4 * t)) & 15u, e = smu[oEX + p * G];
+                    if (e != 0 && e <= now) { free_mask |= 1u << p; smi[oID + p * G] = -1; smu[oEX + p * G] = 0; continue; }
+                    nord |= p << (4 * w); ++w;
+                    if (e && e < next_exp) next_exp = e;
+                }
+                ord = nord; c = w;
+                for (uint32_t t = 0; t < c; ++t) {                           // re-sum the cached terms, slot order
+                    const uint32_t p = (ord >> (4 * t)) & 15u;
+                    float s = 0.0f;
+                    for (uint32_t u = 0; u < c; ++u)
+                        if (u != t) s = __fadd_rn(s, sm[oPT + (p * R + ((ord >> (4 * u)) & 15u)) * G]);
+                    sm[oPA + p * G] = s;
+                }
+            }
+            if (kg + kAhead < g.n) issue(kl + kAhead, kg + kAhead);
+            cp_async_commit();
+
+            uint32_t key_hi = 0xffffffffu;
+            float mean = 0.0f, mu_inc = 0.0f;
+            if (owner && c < R) {                                            // what-if: residents + the arrival
+                float tot = 0.0f;
+                for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {
+                    const uint32_t p = o & 15u;
+                    const uint32_t ti = term_index(kg, p);
+                    const uint32_t i0 = ti & 0x7fffffffu;
+                    const float to = sm[i0];                                  // P[id][inc]
+                    const float from = sm[i0 + ((ti >> 31) ? 1u : GR)];       // P[inc][id]
+                    tot = __fadd_rn(tot, __fadd_rn(sm[oPA + p * G], to));
+                    mu_inc = __fadd_rn(mu_inc, from);
+                }
+                tot = __fadd_rn(tot, mu_inc);
+                mean = __fdiv_rn(tot, (float)(c + 1));
+                if (mean < g.lambda) key_hi = __float_as_uint(mean);         // Algorithm 2 line 7; mean >= 0: bits order
+            }
+            const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
+            const uint32_t best_lo = __reduce_min_sync(0xffffffffu, (key_hi == best_hi && key_hi != 0xffffffffu) ? gpu : 0xffffffffu);
+            if (lane == 0) s_key[k & 1][wid] = ((unsigned long long)best_hi << 32) | best_lo;
+            cp_async_wait<kAhead - 1>();                                     // this thread's share of arrival k+1 landed
+            __syncthreads();
+            unsigned long long best = s_key[k & 1][0];
+            for (uint32_t w = 1; w < nwarps; ++w) {
+                const unsigned long long o = s_key[k & 1][w];
+                best = o < best ? o : best;
+            }
+            // results stay in shared memory until the chunk ends: a global store inside the loop would
+            // have to complete before every barrier
+            if (best == kNoGpu) {
+                if (tid == 0) { smi[oOUT + k] = -1; sm[oOUT + kArrChunk + k] = 0.0f; sm[oOUT + 2 * kArrChunk + k] = 0.0f; }
+            } else if (owner && gpu == (uint32_t)(best & 0xffffffffu)) {
+                const uint32_t pn = __ffs(free_mask) - 1u;                   // lowest free physical slot
+                free_mask &= ~(1u << pn);
+                for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {         // the what-if sums become the cached ones
+                    const uint32_t p = o & 15u;
+                    const uint32_t ti = term_index(kg, p);
+                    const uint32_t i0 = ti & 0x7fffffffu;
+                    const float to = sm[i0], from = sm[i0 + ((ti >> 31) ? 1u : GR)];
+                    sm[oPA + p * G] = __fadd_rn(sm[oPA + p * G], to);
+                    sm[oPT + (p * R + pn) * G] = to;
+                    sm[oPT + (pn * R + p) * G] = from;
+                }
+                sm[oPT + (pn * R + pn) * G] = 0.0f;
+                sm[oPA + pn * G] = mu_inc;
+                smi[oID + pn * G] = smi[oARR + kl];
+                const uint32_t life = (uint32_t)smi[oLIFE + k];
+                const uint32_t e = life ? now + life : 0u;
+                smu[oEX + pn * G] = e;
+                smi[oBI + pn * G] = (int32_t)(kg + 1);
+                if (e && e < next_exp) next_exp = e;
+                ord |= pn << (4 * c);
+                ++c;
+                smi[oOUT + k] = (int32_t)gpu;
+                sm[oOUT + kArrChunk + k] = mean;
+                sm[oOUT + 2 * kArrChunk + k] = mu_inc;
+            }
+        }
+        __syncthreads();
+        for (uint32_t i = tid; i < kn; i += blockDim.x) {
+            g.gpu_out[k0 + i] = smi[oOUT + i];
+            if (g.mean_out) g.mean_out[k0 + i] = sm[oOUT + kArrChunk + i];
+            if (g.mu_arr_out) g.mu_arr_out[k0 + i] = sm[oOUT + 2 * kArrChunk + i];
+        }
+    }
+    cp_async_wait<0>();
+    if (owner) {                                                             // write back in arrival order
+        g.count[gpu] = c;
+        for (uint32_t t = 0; t < R; ++t) {
+            const uint32_t p = (ord >> (4 * t)) & 15u;
+            g.ids[gpu * R + t] = t < c ? smi[oID + p * G] : -1;
+            g.expiry[gpu * R + t] = t < c ? smu[oEX + p * G] : 0u;
+        }
+    }
+    if (tid == 0) *g.tick = tick0 + g.n;
+}
+
 }  // namespace roomie
 
 using namespace roomie;
@@ -317,6 +541,23 @@ extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_
     a.ids = state->ids; a.expiry = state->expiry; a.count = state->count; a.tick = state->tick;
     a.arr_id = arr_id; a.arr_life = arr_life; a.n = n; a.lambda = opts->lambda;
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t GR = (size_t)a.G * a.R;
+    const size_t fast_bytes = GR * 4 * 4 + GR * a.R * 4 + 4 * 2 * GR * 4 + kYoungRing * kAhead * 2 * 4 +
+                              (5 * kArrChunk + 2 * kAhead) * sizeof(int32_t);
+    if (a.R <= 8 && fast_bytes <= 160 * 1024) {
+        // up to 8 slots per GPU: matrix elements are fetched three arrivals ahead
+        a.matrix_mode = 1; a.pair_cache = 1;
+        a.gpus_per_warp = 32;
+        const uint32_t threads = 32 * ((a.G + a.gpus_per_warp - 1) / a.gpus_per_warp + 1);   // + the helper warp
+        auto kern = place_fast_kernel;
+        if (fast_bytes > 48 * 1024)
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast_bytes));
+        kern<<<1, threads, fast_bytes, st>>>(a);
+        note_launch();
+        ROOMIE_CUDA_OK(cudaGetLastError());
+        return ROOMIE_OK;
+    }
     size_t state_bytes = (size_t)a.G * a.R * 12 + 2 * kArrChunk * sizeof(int32_t);
     const size_t pair_bytes = (size_t)a.G * a.R * a.R * sizeof(float);
     a.pair_cache = pair_bytes <= 64 * 1024;
@@ -329,11 +570,10 @@ extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_
     else a.matrix_mode = 2;
     uint32_t threads = ((a.G + 31) / 32) * 32;
     if (a.matrix_mode == 1 && threads < 128) threads = 128;          // more lanes to issue the prefetch
-    auto kern = a.R <= 4 ? place_kernel<4> : a.R <= 8 ? place_kernel<8> : a.R <= 16 ? place_kernel<16>
-                                                                                   : place_kernel<0>;
+    auto kern = a.R <= 16 ? place_kernel<16> : place_kernel<0>;
     if (smem > 48 * 1024)
         ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<1, threads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+    kern<<<1, threads, smem, st>>>(a);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;
