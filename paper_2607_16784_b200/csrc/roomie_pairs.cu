@@ -210,8 +210,8 @@ struct TileArgs {
 };
 
 // Shared-memory layout of one tile.  The tile's A records sit at unified indices 0, 1, 2, ... and
-// its B records at kTileLoad-1, kTileLoad-2, ... (the two runs never meet: together they hold at
-// most kTileLoad records).  Records are padded by one slot after every 8 so that the lanes of a
+// its B records at kTop, kTop-1, ... (the two runs never meet: together they hold at most
+// kTileLoad <= kTop + 1 records).  Records are padded by one slot after every 8 so that the lanes of a
 // warp, whose positions on the merge path are about 8 records apart, fall into different bank
 // groups; the search keys (end ticks) live in their own array with one pad word per 32 so that
 // the binary-search probes of a warp do not collide either.  Both paddings are linear in the
@@ -221,8 +221,10 @@ struct TileArgs {
 __device__ __forceinline__ uint32_t rec_slot(uint32_t i) { return i + (i >> 3); }
 __device__ __forceinline__ uint32_t key_slot(uint32_t i) { return i + (i >> 5); }
 constexpr int kTileLoad = kTileItems + 2;                               // one look-ahead record per side
-constexpr int kRecSlots = kTileLoad + (kTileLoad >> 3) + 2;
-constexpr int kKeySlots = kTileLoad + (kTileLoad >> 5) + 2;
+constexpr int kTop = ((kTileLoad + 31) / 32) * 32 + 31;                  // unified index of B[0]; = 31 mod 32 so that
+                                                                         // a warp's descending run starts on a pad boundary
+constexpr int kRecSlots = kTop + (kTop >> 3) + 2;
+constexpr int kKeySlots = kTop + (kTop >> 5) + 2;
 constexpr int kStageBatch = 6;                                           // global loads in flight per thread
 constexpr int kStageRounds = (kTileLoad + kTileThreads * kStageBatch - 1) / (kTileThreads * kStageBatch);
 
@@ -260,7 +262,7 @@ __device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32
                                            uint4* s_rec, int32_t* s_key) {
     // thread t handles records t, t + 128, ...; 128 is a multiple of 8 and 32, so both paddings
     // advance by a constant per trip
-    const uint32_t i0 = kDir > 0 ? threadIdx.x : (uint32_t)(kTileLoad - 1) - threadIdx.x;
+    const uint32_t i0 = kDir > 0 ? threadIdx.x : (uint32_t)kTop - threadIdx.x;
     uint4* rp = s_rec + rec_slot(i0);
     int32_t* kp = s_key + key_slot(i0);
     constexpr int kRecStep = kDir * (kTileThreads + kTileThreads / 8);
@@ -297,13 +299,16 @@ __device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32
         dj = fmaf(tw, fb, dj);                                                                         \
         if (kWithV) V += hit ? (unsigned long long)(uint32_t)ov : 0ull;                                \
         ties += (Ea == Eb) ? 1u : 0u;                                                                  \
-        if (Ea <= Eb) {                                                                                \
-            ++x; ra = s_rec[rec_slot(x)];                                                              \
-            wslack_a = ra.z >> kWarpShift; fa = small_int_to_float(wconst - wslack_a);                 \
+        /* the kernel that ends first is replaced by its model's next one: a single load for the   */  \
+        /* whole warp, whichever side each lane advances                                           */  \
+        const bool adv_a = Ea <= Eb;                                                                   \
+        x += adv_a ? 1u : 0u;                                                                          \
+        ib -= adv_a ? 0u : 1u;                                                                         \
+        const uint4 r = s_rec[rec_slot(adv_a ? x : ib)];                                               \
+        if (adv_a) {                                                                                   \
+            ra = r; wslack_a = r.z >> kWarpShift; fa = small_int_to_float(wconst - wslack_a);          \
         } else {                                                                                       \
-            --ib; rb = s_rec[rec_slot(ib)];                                                            \
-            const uint32_t wb = rb.z >> kWarpShift;                                                    \
-            wsum_b = wb + wconst; fb = small_int_to_float(wb);                                         \
+            rb = r; wsum_b = (r.z >> kWarpShift) + wconst; fb = small_int_to_float(r.z >> kWarpShift); \
         }                                                                                              \
     }
 
@@ -336,14 +341,14 @@ __global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArg
         uint32_t ties = 0;
         if (diag < len) {
             // this thread's start point on the tile's merge path (A first on equal end times):
-            // B record y sits at unified index kTileLoad - 1 - y
+            // B record y sits at unified index kTop - y
             uint32_t lo = diag > d.cntB ? diag - d.cntB : 0u, hi = diag < d.cntA ? diag : d.cntA;
-            const uint32_t btop = (uint32_t)kTileLoad - diag;              // index of B[diag - 1 - mid] is btop + mid
+            const uint32_t btop = (uint32_t)(kTop + 1) - diag;             // index of B[diag - 1 - mid] is btop + mid
             while (lo < hi) {
                 const uint32_t mid = (lo + hi) >> 1;
                 if (s_key[key_slot(mid)] <= s_key[key_slot(btop + mid)]) lo = mid + 1; else hi = mid;
             }
-            uint32_t x = lo, ib = (uint32_t)(kTileLoad - 1) - (diag - lo);
+            uint32_t x = lo, ib = (uint32_t)kTop - (diag - lo);
             uint4 ra = s_rec[rec_slot(x)], rb = s_rec[rec_slot(ib)];
             uint32_t wslack_a = ra.z >> kWarpShift, wsum_b = (rb.z >> kWarpShift) + wconst;
             float fa = small_int_to_float(wconst - wslack_a), fb = small_int_to_float(rb.z >> kWarpShift);
