@@ -183,6 +183,30 @@ int roomie_pair_interference(const roomie_library *lib /* host */, uint32_t a, u
                              const roomie_pair_detail *detail, void *workspace, size_t workspace_bytes,
                              void *stream);
 
+/* roomie_pair_interference without a workspace argument (the paper has no counterpart: this is
+ * a deployment aid).  It is meant for callers that cannot obtain device memory of their own:
+ * a placement controller living beside an inference runtime whose allocator already owns the
+ * whole device, a plug-in that is handed raw device pointers but no allocator, or a service
+ * loop in which a cudaMalloc would stall every stream of the device.  The scratch the walk
+ * needs lives in a fixed array of ROOMIE_STATIC_SCRATCH_BYTES inside the library image; every
+ * GPU that loads the library holds that array until the process exits.  Inputs and outputs are
+ * still the caller's.  The call allocates nothing: no cudaMalloc, no cudaFree, no allocating
+ * library routine.
+ *   - Same arguments, results and errors as roomie_pair_interference; a pair whose scratch need
+ *     exceeds the array (very long profiles combined with many alignments) is refused with
+ *     ROOMIE_ERR_CAPACITY and nothing is enqueued.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress,
+ *     with that device current) and remembers it; make that first call during start-up, before
+ *     any stream capture begins.
+ *   - All calls on a device share the one array.  Each call clears what it needs cleared, so
+ *     calls issued one after the other on a stream are independent, but two calls whose GPU
+ *     work overlaps (different streams without an ordering between them, or different host
+ *     threads) race on the array and give wrong results: serialise them. */
+#define ROOMIE_STATIC_SCRATCH_BYTES (1u << 20)
+int roomie_pair_interference_static(const roomie_library *lib /* host */, uint32_t a, uint32_t b,
+                                    const roomie_opts *opts /* host */, float *out2, uint64_t *evals_out,
+                                    const roomie_pair_detail *detail, void *stream);
+
 /* Algorithm 1, outer loops, given the pairwise terms (performance_drop(M)), batched over
  * n_sets independent model sets.  Set s is M = resident_ids[s*max_residents + 0..count[s])
  * followed by incoming[s] (profile ids, duplicates allowed = replicas).

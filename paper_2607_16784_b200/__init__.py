@@ -10,6 +10,6 @@ There is no CPU fallback: importing this package without the compiled library ra
 """
 from .roomie import (  # noqa: F401
     GpuSpec, Library, ClusterState, RoomieError, TIMELINE, LOCKSTEP,
-    occupancy, library_build, pair_workspace_bytes, pair_matrix, pair_interference,
+    occupancy, library_build, pair_workspace_bytes, pair_matrix, pair_interference, pair_interference_static,
     multi_estimate, place, launch_count, reset_launch_count, profile_enable, profile_walk_ms, lib_path, EXPORTS,
 )

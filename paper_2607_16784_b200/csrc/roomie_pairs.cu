@@ -695,6 +695,33 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
 
 using namespace roomie;
 
+// ---------------------------------------------------------------------------------------
+// Scratch for roomie_pair_interference_static: part of the library image, so every GPU that
+// loads the library keeps it until the process exits.  Host code must not pass the symbol
+// itself to a kernel (on the host its name is only a handle): the device address is looked up
+// once per device with cudaGetSymbolAddress while that device is current.
+// ---------------------------------------------------------------------------------------
+namespace roomie {
+constexpr size_t kStaticScratchBytes = ROOMIE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+constexpr int kMaxDevices = 64;
+static void* g_static_scratch_addr[kMaxDevices];       // device address per device ordinal, 0 = not looked up yet
+
+static int static_scratch_for_current_device(void** out) {
+    int dev = 0;
+    ROOMIE_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return ROOMIE_ERR_INVALID_ARG;
+    void* p = __atomic_load_n(&g_static_scratch_addr[dev], __ATOMIC_ACQUIRE);
+    if (!p) {
+        ROOMIE_CUDA_OK(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return ROOMIE_ERR_CUDA;
+        __atomic_store_n(&g_static_scratch_addr[dev], p, __ATOMIC_RELEASE);   // same value from every thread
+    }
+    *out = p;
+    return ROOMIE_OK;
+}
+}  // namespace roomie
+
 extern "C" size_t roomie_pair_workspace_bytes(const roomie_library* lib, const roomie_opts* opts,
                                               uint64_t pair_begin, uint64_t pair_end) {
     if (check_lib(lib, opts) != ROOMIE_OK) return 0;
@@ -763,4 +790,28 @@ extern "C" int roomie_pair_interference(const roomie_library* lib, uint32_t a, u
     PairSet ps;
     ps.pair_begin = 0; ps.n_pairs = 1; ps.explicit_pair = 1; ps.a = a; ps.b = b;
     return run_batch(lib, opts, ps, slots, need, out2, evals_out, detail, static_cast<unsigned char*>(workspace), st);
+}
+
+extern "C" int roomie_pair_interference_static(const roomie_library* lib, uint32_t a, uint32_t b,
+                                               const roomie_opts* opts, float* out2, uint64_t* evals_out,
+                                               const roomie_pair_detail* detail, void* stream) {
+    int rc = check_lib(lib, opts);
+    if (rc != ROOMIE_OK) return rc;
+    if (!out2 || a >= lib->num_profiles || b >= lib->num_profiles) return ROOMIE_ERR_INVALID_ARG;
+    uint32_t slots;
+    rc = slots_for(lib, opts, true, a, b, slots);
+    if (rc != ROOMIE_OK) return rc;
+    Need need;
+    batch_need(lib, opts, true, a, b, 0, 1, slots, need);
+    if (bytes_for(need) > kStaticScratchBytes) return ROOMIE_ERR_CAPACITY;   // beyond the built-in scratch
+    void* scratch = nullptr;
+    rc = static_scratch_for_current_device(&scratch);
+    if (rc != ROOMIE_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), st));
+    PairSet ps;
+    ps.pair_begin = 0; ps.n_pairs = 1; ps.explicit_pair = 1; ps.a = a; ps.b = b;
+    // run_batch zeroes the tile counter at the head of the scratch; everything else in it is
+    // written by the plan kernel before it is read, so the previous call's contents do not matter
+    return run_batch(lib, opts, ps, slots, need, out2, evals_out, detail, static_cast<unsigned char*>(scratch), st);
 }

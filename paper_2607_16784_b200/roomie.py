@@ -16,6 +16,7 @@ TIMELINE, LOCKSTEP = 0, 1
 EXPORTS = [
     "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
+    "roomie_pair_interference_static",
     "roomie_multi_estimate", "roomie_place", "roomie_strerror", "roomie_last_cuda_error",
     "roomie_launch_count", "roomie_reset_launch_count", "roomie_profile_enable", "roomie_profile_walk_ms",
 ]
@@ -45,6 +46,8 @@ def _load():
                                        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     dll.roomie_pair_interference.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    dll.roomie_pair_interference_static.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
+                                                    C.c_void_p, C.c_void_p, C.c_void_p]
     dll.roomie_occupancy.argtypes = [C.c_void_p] * 4
     dll.roomie_library_build.argtypes = [C.c_void_p] * 5
     dll.roomie_multi_estimate.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -245,14 +248,9 @@ def pair_matrix(lib: Library, *, mode=TIMELINE, n_align=1, start_filter=0, pair_
     return out, evals
 
 
-def pair_interference(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1, start_filter=0,
-                      detail_capacity=0, workspace=None, stream=None):
-    """roomie_pair_interference: one ordered pair.  Returns a dict with P_ab, P_ba (float32 [2] tensor
-    `P2`), evals and, when detail_capacity > 0, the per-alignment arrays."""
-    dev = lib.records.device
+def _pair_outputs(dev, detail_capacity):
     out2 = torch.zeros(2, dtype=torch.float32, device=dev)
     evals = torch.zeros(1, dtype=torch.int64, device=dev)
-    o = _opts(mode, n_align, start_filter)
     res = dict(P2=out2, evals=evals)
     det = None
     if detail_capacity > 0:
@@ -267,16 +265,37 @@ def pair_interference(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1,
         det = _Detail(cap, res["n_kept"].data_ptr(), res["s_i"].data_ptr(), res["s_j"].data_ptr(),
                       res["delta_i"].data_ptr(), res["delta_j"].data_ptr(), res["V"].data_ptr(),
                       res["evals_c"].data_ptr())
+    return res, det
+
+
+def pair_interference(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1, start_filter=0,
+                      detail_capacity=0, workspace=None, stream=None):
+    """roomie_pair_interference: one ordered pair.  Returns a dict with P_ab, P_ba (float32 [2] tensor
+    `P2`), evals and, when detail_capacity > 0, the per-alignment arrays."""
+    dev = lib.records.device
+    o = _opts(mode, n_align, start_filter)
+    res, det = _pair_outputs(dev, detail_capacity)
     if workspace is None:
-        # a single pair never needs more than the whole triangle; size it from the pair's own row
         qa = int(lib.offsets_host[a + 1] - lib.offsets_host[a])
         qb = int(lib.offsets_host[b + 1] - lib.offsets_host[b])
         slots = (qa * qb) if n_align == 0 else n_align * n_align
         tiles = slots * ((qa + qb) // 2048 + 2)
         workspace = _workspace(4096 + slots * 16 + tiles * 64, dev)
-    _check(_dll.roomie_pair_interference(C.byref(lib.c), a, b, C.byref(o), _ptr(out2), _ptr(evals),
+    _check(_dll.roomie_pair_interference(C.byref(lib.c), a, b, C.byref(o), _ptr(res["P2"]), _ptr(res["evals"]),
                                          C.byref(det) if det is not None else None, _ptr(workspace),
                                          workspace.numel(), _stream(stream)), "roomie_pair_interference")
+    return res
+
+
+def pair_interference_static(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1, start_filter=0,
+                             detail_capacity=0, stream=None):
+    """roomie_pair_interference_static: the same result computed in the library's built-in scratch
+    array - for callers that cannot allocate device memory.  Calls that overlap on the GPU race."""
+    o = _opts(mode, n_align, start_filter)
+    res, det = _pair_outputs(lib.records.device, detail_capacity)
+    _check(_dll.roomie_pair_interference_static(C.byref(lib.c), a, b, C.byref(o), _ptr(res["P2"]),
+                                                _ptr(res["evals"]), C.byref(det) if det is not None else None,
+                                                _stream(stream)), "roomie_pair_interference_static")
     return res
 
 
