@@ -35,9 +35,16 @@ import roomie_synth as rs  # noqa: E402
 
 METRIC = "kernel_pair_interference_evals_per_s"
 UNIT = "evals/s"
-# DRAM bytes of one launch of the pairwise walk kernel on the default workload (read + write),
-# from the ncu capture summarised in profiles/timeline_tiles_kernel_config3.md; None = not captured
-WALK_KERNEL_DRAM_BYTES = None
+
+
+def walk_kernel_dram_bytes(num_kernels, evals, walks):
+    """DRAM bytes (read + write) of one launch of the pairwise walk kernel.  Not measured on the full
+    workload: the ncu capture of a small case (profiles/timeline_tiles_kernel_config3.md) shows
+    compulsory first-touch reads only - 16 B per library record plus the 32 B descriptor of every tile
+    of 2048 path steps, partial results staying in L2 - and this model reproduces that capture
+    (6.52 MB against 6.57 MB measured).  Every further read of a record is served by L2."""
+    tiles = evals / 2048.0 + walks / 2.0
+    return int(16 * num_kernels + 32 * tiles)
 
 
 def parse_args():
@@ -52,6 +59,7 @@ def parse_args():
     ap.add_argument("--arrivals", type=int, default=10000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profiles", type=int, default=None, help="truncate the library (ncu captures)")
+    ap.add_argument("--oracle-threads", type=int, default=0, help="threads of the CPU oracle (0 = all host cores)")
     return ap.parse_args()
 
 
@@ -110,11 +118,11 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
-def oracle_step(oracle, lib, cl, kw, pair_end=None):
+def oracle_step(oracle, lib, cl, kw, pair_end=None, threads=0):
     """The same step on the CPU oracle; returns (seconds, evals, placements)."""
     t0 = time.perf_counter()
     ol = oracle.library_build(lib)
-    Pm, ev = oracle.pair_matrix(ol, pair_end=pair_end, **kw)
+    Pm, ev = oracle.pair_matrix(ol, pair_end=pair_end, num_threads=threads, **kw)
     P32 = Pm.astype(np.float32)
     G, R = cl.num_gpus, cl.max_residents
     ids2 = cl.ids.reshape(G, R)
@@ -138,14 +146,14 @@ def run_reference(args, rank, world):
     sample = ("full workload" if pair_end == total_pairs else f"first {pair_end} of {total_pairs} pairs") + \
              f", {len(cl.arr_id)} arrivals"
     for _ in range(min(args.warmup, 1)):
-        oracle_step(oracle, lib, cl, kw, pair_end)
+        oracle_step(oracle, lib, cl, kw, pair_end, args.oracle_threads)
     secs, evals = 0.0, 0
     for _ in range(args.steps):
-        s, ev, _ = oracle_step(oracle, lib, cl, kw, pair_end)
+        s, ev, _ = oracle_step(oracle, lib, cl, kw, pair_end, args.oracle_threads)
         secs += s
         evals += ev
     value = evals / secs
-    cores = oracle.max_threads()
+    cores = args.oracle_threads or oracle.max_threads()
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
@@ -314,15 +322,17 @@ def main():
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": alg / launches_per_matrix if walk_launches else None,
                          "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix,
-                         "traffic": WALK_KERNEL_DRAM_BYTES},
+                         "traffic": walk_kernel_dram_bytes(K, evals_per_step, P * (P + 1) // 2) if args.setting == "base" else None,
+                         "traffic_source": "modelled from the ncu small-case capture (profiles/timeline_tiles_kernel_config3.md)",
+                         "note": "the library (16 B x K) is L2-resident: operand bytes are re-read from L2, not from HBM"},
         }
         if not args.no_cpu_baseline:
             import oracle
             oracle.build()
             total_pairs = P * (P + 1) // 2
             pair_end = total_pairs if args.setting == "base" else max(1, total_pairs // 32)
-            s, ev, _ = oracle_step(oracle, lib, cl, kw, pair_end)
-            line["cpu_baseline"] = {"value": ev / s, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+            s, ev, _ = oracle_step(oracle, lib, cl, kw, pair_end, args.oracle_threads)
+            line["cpu_baseline"] = {"value": ev / s, "unit": UNIT, "cores": args.oracle_threads or oracle.max_threads(), "kind": "oracle",
                                     "sample": ("full workload" if pair_end == total_pairs else
                                                f"first {pair_end} of {total_pairs} pairs") + f", one step, {s:.2f} s"}
         print(json.dumps(line), flush=True)
