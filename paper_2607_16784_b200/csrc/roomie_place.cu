@@ -292,17 +292,22 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
 //   - every resident sits in a fixed *physical* slot; the arrival order of a GPU's residents is a
 //     packed nibble list in a register, so a departure moves no shared-memory data and copies in
 //     flight never have to follow a resident;
-//   - at arrival j each thread issues cp.async for the 2 matrix elements per resident that
-//     arrival j+3 will need, into a 4-deep ring indexed by physical slot;
-//   - a resident younger than 3 arrivals is not covered by the ring (it was placed after the
-//     fetch was issued); its terms depend only on the arrival stream (P[arr_{j-d}][arr_j] and the
-//     transpose, d = 1..3) and are fetched by six designated threads on the same schedule.
-// The critical path per arrival is shared-memory reads, 2c+2 float adds, one division, two
-// redux steps and one barrier.
+//   - the CTA is split into owner warps (one lane per modelled GPU: departures, what-if sums,
+//     argmin, winner update) and as many fetch warps.  While arrival j is decided, the fetch lane
+//     of a GPU issues cp.async for the two matrix elements per resident that arrival j+3 will
+//     need, into a 4-deep ring indexed by physical slot; it reads the GPU's order list from a
+//     64-bit word the owner publishes whenever the list changes;
+//   - a resident placed fewer than 5 arrivals ago may have been missed by those fetches (they
+//     were issued before, or while, it was placed); its terms depend only on the arrival stream
+//     (P[arr_{j-d}][arr_j] and the transpose, d = 1..4) and are fetched on the same schedule.
+// The owners' critical path per arrival is shared-memory reads, 2c+2 float adds, one division,
+// two redux steps and one barrier; no global memory access and no copy wait.
 // ---------------------------------------------------------------------------------------
 constexpr int kAhead = 3;                     // arrivals fetched ahead
+constexpr int kYoungD = kAhead + 1;           // residents this young read the arrival-to-arrival terms
 constexpr int kYoungRing = 8;                 // ring depth of the arrival-to-arrival terms
 constexpr int kYoungInit = -(1 << 30);        // birth index of initial residents
+constexpr int kLead = kYoungD;                // arrival ids staged before / after a chunk
 
 __device__ __forceinline__ void cp_async_4_s(uint32_t smem_addr, const void* gmem_src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(smem_addr), "l"(gmem_src) : "memory");
@@ -315,25 +320,25 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
     uint32_t* smu = reinterpret_cast<uint32_t*>(sm);
     const uint32_t G = g.G, R = g.R, P = g.P, GR = G * R;
     const uint32_t tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = blockDim.x >> 5;
-    // GPUs are spread over the warps (gpw per warp, low lanes) so that the serial sections of an
-    // arrival - a departure on one GPU, the winner's update on another - run in different warps;
-    // the last warp owns no GPU and fetches the arrival-to-arrival terms
-    const uint32_t gpw = g.gpus_per_warp;
-    const uint32_t gpu = wid * gpw + lane;
-    const bool helper = wid == nwarps - 1;
+    const uint32_t n_owner_warps = nwarps >> 1;
+    const bool fetcher = wid >= n_owner_warps;
+    const uint32_t gpu = (fetcher ? wid - n_owner_warps : wid) * 32 + lane;
+    const bool has_gpu = gpu < G;
+    const bool owner = !fetcher && has_gpu;
     // word offsets of the regions; per-GPU arrays are [slot][gpu]
     const uint32_t oID = gpu, oEX = GR + gpu, oPA = 2 * GR + gpu, oBI = 3 * GR + gpu;
     const uint32_t oPT = 4 * GR + gpu;                    // [slot][slot][gpu]
     const uint32_t oRING = 4 * GR + GR * R + gpu;         // [4][2][slot][gpu]
-    const uint32_t oYOUNG = 4 * GR + GR * R + 8 * GR;     // [kYoungRing][kAhead][2]
-    const uint32_t oARR = oYOUNG + kYoungRing * kAhead * 2;   // ids [kArrChunk + 2 kAhead], then lifetimes [kArrChunk]
-    const uint32_t oLIFE = oARR + kArrChunk + 2 * kAhead;
+    const uint32_t oYOUNG = 4 * GR + GR * R + 8 * GR;     // [kYoungRing][kYoungD][2]
+    const uint32_t oPUB = (oYOUNG + kYoungRing * kYoungD * 2 + 1) & ~1u;   // [G] 64-bit: order list | count << 32
+    const uint32_t oARR = oPUB + 2 * G;                   // ids [kArrChunk + 2 kLead], then lifetimes [kArrChunk]
+    const uint32_t oLIFE = oARR + kArrChunk + 2 * kLead;
     const uint32_t oOUT = oLIFE + kArrChunk;              // decisions of the chunk: gpu, mean, mu_arr [3][kArrChunk]
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(sm);
+    volatile unsigned long long* pub = reinterpret_cast<volatile unsigned long long*>(sm + oPUB);
     __shared__ unsigned long long s_key[2][32];
 
     const float* __restrict__ Pm = g.Pm;
-    const bool owner = !helper && lane < gpw && gpu < G;
 
     // initial state: residents occupy physical slots 0..c-1 in arrival order
     uint32_t c = 0, ord = 0, free_mask = (1u << R) - 1u, next_exp = 0xffffffffu;
@@ -358,59 +363,66 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 if (q != p) s = __fadd_rn(s, sm[oPT + (p * R + q) * G]);
             sm[oPA + p * G] = s;
         }
+        pub[gpu] = (unsigned long long)ord | ((unsigned long long)c << 32);
     }
     const uint32_t tick0 = *g.tick;
 
-    // fetch what arrival a (s_arr index a_local, global index a_global) will need
+    // fetch warps: what arrival a (staged index a_local, global index a_global) will need
     auto issue = [&](uint32_t a_local, uint32_t a_global) {
         const int32_t inc = smi[oARR + a_local];
         const float* row = Pm + (size_t)inc * P;          // P[inc][*]
         const float* col = Pm + inc;                      // P[*][inc]
-        const uint32_t ring = oRING + (a_global & 3u) * 2 * GR;
-        for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {      // c = 0 for threads that own no GPU
-            const uint32_t p = o & 15u;
-            const int32_t id = smi[oID + p * G];
-            cp_async_4_s(sm_base + 4u * (ring + p * G), col + (size_t)id * P);
-            cp_async_4_s(sm_base + 4u * (ring + GR + p * G), row + id);
+        if (has_gpu) {
+            const unsigned long long pv = pub[gpu];       // one 64-bit read: list and count belong together
+            const uint32_t cc = (uint32_t)(pv >> 32);
+            const uint32_t ring = oRING + (a_global & 3u) * 2 * GR;
+            for (uint32_t t = 0, o = (uint32_t)pv; t < cc; ++t, o >>= 4) {
+                const uint32_t p = o & 15u;
+                const int32_t id = smi[oID + p * G];
+                if (id < 0) continue;                     // just departed
+                cp_async_4_s(sm_base + 4u * (ring + p * G), col + (size_t)id * P);
+                cp_async_4_s(sm_base + 4u * (ring + GR + p * G), row + id);
+            }
         }
-        if (helper && lane < 2 * kAhead) {
+        if (wid == n_owner_warps && lane < 2 * kYoungD) {
             const uint32_t d = (lane >> 1) + 1, dir = lane & 1u;
             if (a_local >= d) {
                 const int32_t old = smi[oARR + a_local - d];
-                cp_async_4_s(sm_base + 4u * (oYOUNG + ((a_global & (kYoungRing - 1)) * kAhead + (d - 1)) * 2 + dir),
+                cp_async_4_s(sm_base + 4u * (oYOUNG + ((a_global & (kYoungRing - 1)) * kYoungD + (d - 1)) * 2 + dir),
                              dir == 0 ? col + (size_t)old * P : row + old);
             }
         }
     };
-    // word index of the term between the arrival kg and the resident in physical slot p:
-    // young residents read the arrival-to-arrival terms, the others the ring
-    auto term_index = [&](uint32_t kg, uint32_t p) -> uint32_t {
-        const uint32_t d1 = (uint32_t)((int32_t)(kg + 1) - smi[oBI + p * G]) - 1u;     // arrivals since placed, minus 1
-        const uint32_t iy = oYOUNG + ((kg & (kYoungRing - 1)) * kAhead + d1) * 2;
-        const uint32_t ir = oRING + (kg & 3u) * 2 * GR + p * G;
-        return d1 < (uint32_t)kAhead ? (iy | 0x80000000u) : ir;                        // top bit: young
-    };
 
     for (uint32_t k0 = 0; k0 < g.n; k0 += kArrChunk) {
         const uint32_t kn = min(kArrChunk, g.n - k0);
-        // stage arrival ids [k0 - kAhead, k0 + kn + kAhead) and lifetimes [k0, k0 + kn)
+        // stage arrival ids [k0 - kLead, k0 + kn + kLead) and lifetimes [k0, k0 + kn)
         __syncthreads();
-        for (uint32_t i = tid; i < kn + 2 * kAhead; i += blockDim.x) {
-            const long long gi = (long long)k0 + i - kAhead;
+        for (uint32_t i = tid; i < kn + 2 * kLead; i += blockDim.x) {
+            const long long gi = (long long)k0 + i - kLead;
             smi[oARR + i] = (gi >= 0 && gi < (long long)g.n) ? g.arr_id[gi] : 0;
         }
         for (uint32_t i = tid; i < kn; i += blockDim.x) smi[oLIFE + i] = (int32_t)g.arr_life[k0 + i];
         __syncthreads();
         if (k0 == 0) {                                                      // prime: arrivals 0 .. kAhead-1
-            for (uint32_t a = 0; a < (uint32_t)kAhead; ++a) {
-                if (a < g.n) issue(a + kAhead, a);
-                cp_async_commit();
+            if (fetcher) {
+                for (uint32_t a = 0; a < (uint32_t)kAhead; ++a) {
+                    if (a < g.n) issue(a + kLead, a);
+                    cp_async_commit();
+                }
+                cp_async_wait<kAhead - 1>();
             }
-            cp_async_wait<kAhead - 1>();
             __syncthreads();
         }
         for (uint32_t k = 0; k < kn; ++k) {
-            const uint32_t kg = k0 + k, now = tick0 + kg, kl = k + kAhead;  // global index, tick, index into the staged ids
+            const uint32_t kg = k0 + k, now = tick0 + kg, kl = k + kLead;   // global index, tick, index into the staged ids
+            if (fetcher) {
+                if (kg + kAhead < g.n) issue(kl + kAhead, kg + kAhead);
+                cp_async_commit();
+                cp_async_wait<kAhead - 1>();                                 // arrival k+1's terms have landed
+                __syncthreads();
+                continue;
+            }
             if (owner && next_exp <= now) {                                  // departures: drop from the order list
                 uint32_t w = 0, nord = 0;
                 next_exp = 0xffffffffu;
@@ -421,6 +433,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                     if (e && e < next_exp) next_exp = e;
                 }
                 ord = nord; c = w;
+                pub[gpu] = (unsigned long long)ord | ((unsigned long long)c << 32);
                 for (uint32_t t = 0; t < c; ++t) {                           // re-sum the cached terms, slot order
                     const uint32_t p = (ord >> (4 * t)) & 15u;
                     float s = 0.0f;
@@ -429,19 +442,20 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                     sm[oPA + p * G] = s;
                 }
             }
-            if (kg + kAhead < g.n) issue(kl + kAhead, kg + kAhead);
-            cp_async_commit();
-
+            // terms of arrival kg: ring (by physical slot) or, for young residents, arrival-to-arrival
+            const uint32_t ring_k = oRING + (kg & 3u) * 2 * GR;
+            const uint32_t young_k = oYOUNG + (kg & (kYoungRing - 1)) * kYoungD * 2;
             uint32_t key_hi = 0xffffffffu;
             float mean = 0.0f, mu_inc = 0.0f;
             if (owner && c < R) {                                            // what-if: residents + the arrival
                 float tot = 0.0f;
                 for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {
                     const uint32_t p = o & 15u;
-                    const uint32_t ti = term_index(kg, p);
-                    const uint32_t i0 = ti & 0x7fffffffu;
+                    const uint32_t d1 = (uint32_t)((int32_t)kg - smi[oBI + p * G]);   // arrivals since placed, minus 1 (huge if old)
+                    const bool young = d1 < (uint32_t)kYoungD;
+                    const uint32_t i0 = young ? young_k + 2 * d1 : ring_k + p * G;
                     const float to = sm[i0];                                  // P[id][inc]
-                    const float from = sm[i0 + ((ti >> 31) ? 1u : GR)];       // P[inc][id]
+                    const float from = sm[i0 + (young ? 1u : GR)];            // P[inc][id]
                     tot = __fadd_rn(tot, __fadd_rn(sm[oPA + p * G], to));
                     mu_inc = __fadd_rn(mu_inc, from);
                 }
@@ -452,10 +466,9 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
             const uint32_t best_lo = __reduce_min_sync(0xffffffffu, (key_hi == best_hi && key_hi != 0xffffffffu) ? gpu : 0xffffffffu);
             if (lane == 0) s_key[k & 1][wid] = ((unsigned long long)best_hi << 32) | best_lo;
-            cp_async_wait<kAhead - 1>();                                     // this thread's share of arrival k+1 landed
             __syncthreads();
             unsigned long long best = s_key[k & 1][0];
-            for (uint32_t w = 1; w < nwarps; ++w) {
+            for (uint32_t w = 1; w < n_owner_warps; ++w) {
                 const unsigned long long o = s_key[k & 1][w];
                 best = o < best ? o : best;
             }
@@ -468,9 +481,10 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 free_mask &= ~(1u << pn);
                 for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {         // the what-if sums become the cached ones
                     const uint32_t p = o & 15u;
-                    const uint32_t ti = term_index(kg, p);
-                    const uint32_t i0 = ti & 0x7fffffffu;
-                    const float to = sm[i0], from = sm[i0 + ((ti >> 31) ? 1u : GR)];
+                    const uint32_t d1 = (uint32_t)((int32_t)kg - smi[oBI + p * G]);
+                    const bool young = d1 < (uint32_t)kYoungD;
+                    const uint32_t i0 = young ? young_k + 2 * d1 : ring_k + p * G;
+                    const float to = sm[i0], from = sm[i0 + (young ? 1u : GR)];
                     sm[oPA + p * G] = __fadd_rn(sm[oPA + p * G], to);
                     sm[oPT + (p * R + pn) * G] = to;
                     sm[oPT + (pn * R + p) * G] = from;
@@ -481,10 +495,12 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 const uint32_t life = (uint32_t)smi[oLIFE + k];
                 const uint32_t e = life ? now + life : 0u;
                 smu[oEX + pn * G] = e;
-                smi[oBI + pn * G] = (int32_t)(kg + 1);
+                smi[oBI + pn * G] = (int32_t)(kg + 1);                       // first arrival that sees this resident
                 if (e && e < next_exp) next_exp = e;
                 ord |= pn << (4 * c);
                 ++c;
+                __threadfence_block();                                       // id before the list that names its slot
+                pub[gpu] = (unsigned long long)ord | ((unsigned long long)c << 32);
                 smi[oOUT + k] = (int32_t)gpu;
                 sm[oOUT + kArrChunk + k] = mean;
                 sm[oOUT + 2 * kArrChunk + k] = mu_inc;
@@ -543,13 +559,13 @@ extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t GR = (size_t)a.G * a.R;
-    const size_t fast_bytes = GR * 4 * 4 + GR * a.R * 4 + 4 * 2 * GR * 4 + kYoungRing * kAhead * 2 * 4 +
-                              (5 * kArrChunk + 2 * kAhead) * sizeof(int32_t);
-    if (a.R <= 8 && fast_bytes <= 160 * 1024) {
-        // up to 8 slots per GPU: matrix elements are fetched three arrivals ahead
+    const size_t fast_bytes = GR * 4 * 4 + GR * a.R * 4 + 4 * 2 * GR * 4 + (kYoungRing * kYoungD * 2 + 2) * 4 +
+                              2 * a.G * 4 + (5 * kArrChunk + 2 * kLead) * sizeof(int32_t);
+    if (a.R <= 8 && a.G <= 512 && fast_bytes <= 160 * 1024) {
+        // up to 8 slots per GPU: matrix elements are fetched three arrivals ahead by fetch warps
         a.matrix_mode = 1; a.pair_cache = 1;
         a.gpus_per_warp = 32;
-        const uint32_t threads = 32 * ((a.G + a.gpus_per_warp - 1) / a.gpus_per_warp + 1);   // + the helper warp
+        const uint32_t threads = 2 * 32 * ((a.G + 31) / 32);                 // owner warps + as many fetch warps
         auto kern = place_fast_kernel;
         if (fast_bytes > 48 * 1024)
             ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast_bytes));
