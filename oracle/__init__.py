@@ -222,7 +222,8 @@ class Placement:
     tick: int
 
 
-def place(Pm32, num_gpus, max_residents, ids, expiry, count, tick, arr_id, arr_life, lam) -> Placement:
+def place(Pm32, num_gpus, max_residents, ids, expiry, count, tick, arr_id, arr_life, lam,
+          admit_rule: int = 0, objective: int = 0) -> Placement:
     """Runs the placement stream on copies of the state arrays."""
     Pm32 = np.ascontiguousarray(Pm32, dtype=np.float32)
     P = Pm32.shape[0]
@@ -239,5 +240,6 @@ def place(Pm32, num_gpus, max_residents, ids, expiry, count, tick, arr_id, arr_l
     t = C.c_uint32(int(tick))
     _lib().oracle_place(_p(Pm32), C.c_uint32(P), C.c_uint32(num_gpus), C.c_uint32(max_residents),
                         _p(ids), _p(expiry), _p(count), C.byref(t), _p(arr_id), _p(arr_life),
-                        C.c_uint32(n), C.c_float(lam), _p(gpu), _p(mean), _p(mu_arr), _p(near))
+                        C.c_uint32(n), C.c_float(lam), C.c_int(admit_rule), C.c_int(objective),
+                        _p(gpu), _p(mean), _p(mu_arr), _p(near))
     return Placement(gpu, mean, mu_arr, near, ids, expiry, count, int(t.value))

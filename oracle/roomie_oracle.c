@@ -380,19 +380,29 @@ void oracle_multi_estimate(const float *Pm, uint32_t P, const int32_t *ids, uint
  * admissible GPU with the lowest mean wins, lowest index on ties; no
  * admissible GPU -> -1 (deferred) and nothing is added.
  *
- * near_tie[n] (optional) = 1 when, in the double shadow, the winner's mean
+ * near_tie[n] (optional) = 1 when, in the double shadow, the winner's score
  * is within 1e-5 relative of another candidate's or of lambda: decisions
  * that float rounding of the pairwise matrix could legitimately flip.
+ *
+ * Variants (Section 3.4: the objective "can be easily substituted"; the
+ * comment in Algorithm 2 asks that "no variant has a performance drop beyond
+ * lambda"):
+ *   admit_rule 0: mean drop < lambda (Algorithm 2 as printed), 1: the
+ *                 largest member drop < lambda;
+ *   objective  0: lowest mean drop (as printed), 1: lowest largest member
+ *                 drop, 2: lowest drop of the arriving model.
  * ------------------------------------------------------------------ */
 void oracle_place(const float *Pm, uint32_t P, uint32_t G, uint32_t R,
                   int32_t *ids, uint32_t *expiry, uint32_t *count, uint32_t *tick,
                   const int32_t *arr_id, const uint32_t *arr_life, uint32_t n,
-                  float lambda, int32_t *gpu_out, float *mean_out, float *mu_arr_out,
+                  float lambda, int admit_rule, int objective,
+                  int32_t *gpu_out, float *mean_out, float *mu_arr_out,
                   uint8_t *near_tie)
 {
     float *mu = (float *)malloc(sizeof(float) * (R + 1));
     double *mu64 = (double *)malloc(sizeof(double) * (R + 1));
-    double *mean64_g = (double *)malloc(sizeof(double) * (G ? G : 1));
+    double *admit64_g = (double *)malloc(sizeof(double) * (G ? G : 1));   /* shadow; < 0: no free slot */
+    double *score64_g = (double *)malloc(sizeof(double) * (G ? G : 1));
     for (uint32_t a = 0; a < n; ++a) {
         const uint32_t now = *tick + a;
         for (uint32_t g = 0; g < G; ++g) {                 /* departures */
@@ -407,26 +417,35 @@ void oracle_place(const float *Pm, uint32_t P, uint32_t G, uint32_t R,
             for (uint32_t s = w; s < R; ++s) { ids[g * R + s] = -1; expiry[g * R + s] = 0; }
             count[g] = w;
         }
-        int32_t best = -1; float best_mean = 0.0f, best_mu = 0.0f;
+        int32_t best = -1; float best_mean = 0.0f, best_mu = 0.0f, best_score = 0.0f;
         for (uint32_t g = 0; g < G; ++g) {
-            mean64_g[g] = -1.0;
+            admit64_g[g] = -1.0; score64_g[g] = -1.0;
             if (count[g] >= R) continue;                   /* no free slot */
             float mean; double mean64;
             oracle_multi_estimate(Pm, P, ids + g * R, count[g], arr_id[a], mu, &mean, mu64, &mean64);
-            mean64_g[g] = mean64;
-            if (!(mean < lambda)) continue;                /* Algorithm 2 line 7 */
-            if (best < 0 || mean < best_mean) { best = (int32_t)g; best_mean = mean; best_mu = mu[count[g]]; }
+            float worst = 0.0f; double worst64 = 0.0;
+            for (uint32_t i = 0; i <= count[g]; ++i) {
+                if (mu[i] > worst) worst = mu[i];
+                if (mu64[i] > worst64) worst64 = mu64[i];
+            }
+            const float admit = admit_rule == 1 ? worst : mean;
+            const float score = objective == 1 ? worst : objective == 2 ? mu[count[g]] : mean;
+            admit64_g[g] = admit_rule == 1 ? worst64 : mean64;
+            score64_g[g] = objective == 1 ? worst64 : objective == 2 ? mu64[count[g]] : mean64;
+            if (!(admit < lambda)) continue;               /* Algorithm 2 line 7 */
+            if (best < 0 || score < best_score) {
+                best = (int32_t)g; best_score = score; best_mean = mean; best_mu = mu[count[g]];
+            }
         }
         if (near_tie) {
             uint8_t nt = 0;
-            const double tol = 1e-5;
+            const double tol = 1e-5, lam = (double)lambda;
             for (uint32_t g = 0; g < G; ++g) {
-                if (mean64_g[g] < 0.0) continue;
-                const double x = mean64_g[g];
-                if (fabs(x - (double)lambda) <= tol * fabs((double)lambda)) nt = 1;
-                if (best >= 0 && (int32_t)g != best) {
-                    const double y = mean64_g[best];
-                    if (fabs(x - y) <= tol * fmax(fabs(x), fabs(y))) nt = 1;
+                if (admit64_g[g] < 0.0) continue;
+                if (fabs(admit64_g[g] - lam) <= tol * fabs(lam)) nt = 1;       /* admission within rounding */
+                if (best >= 0 && (int32_t)g != best && admit64_g[g] < lam * (1.0 + tol)) {
+                    const double x = score64_g[g], y = score64_g[best];
+                    if (fabs(x - y) <= tol * fmax(fabs(x), fabs(y))) nt = 1;     /* two candidates within rounding */
                 }
             }
             near_tie[a] = nt;
@@ -441,5 +460,5 @@ void oracle_place(const float *Pm, uint32_t P, uint32_t G, uint32_t R,
         }
     }
     *tick += n;
-    free(mu); free(mu64); free(mean64_g);
+    free(mu); free(mu64); free(admit64_g); free(score64_g);
 }

@@ -62,7 +62,7 @@ def test_hand_placement_example(oracle):
     assert list(run(1, [1, -1], [1], 0.515625).gpu) == [-1]
 
 
-def brute_place(Pm, G, R, ids, expiry, count, arr_id, arr_life, lam):
+def brute_place(Pm, G, R, ids, expiry, count, arr_id, arr_life, lam, admit_rule=0, objective=0):
     """Independent restatement with python lists and float64 means (used only where
     float32 rounding cannot matter: Pm entries are multiples of 1/64)."""
     res = [[(int(ids[g * R + s]), int(expiry[g * R + s])) for s in range(int(count[g]))] for g in range(G)]
@@ -77,8 +77,10 @@ def brute_place(Pm, G, R, ids, expiry, count, arr_id, arr_life, lam):
             M = [i for i, _ in res[g]] + [int(m)]
             mu = [sum(Fraction(float(Pm[a, b])) for j, b in enumerate(M) if j != i) for i, a in enumerate(M)]
             mean = sum(mu) / len(M)
-            if mean < Fraction(lam) and (best_mean is None or mean < best_mean):
-                best, best_mean = g, mean
+            admit = max(mu) if admit_rule == 1 else mean
+            score = max(mu) if objective == 1 else mu[-1] if objective == 2 else mean
+            if admit < Fraction(lam) and (best_mean is None or score < best_mean):
+                best, best_mean = g, score
         out.append(best)
         if best >= 0:
             res[best].append((int(m), n + int(life) if life else 0))
@@ -108,6 +110,45 @@ def test_placement_against_brute_force(oracle, seed):
     for g in range(G):
         assert int(got.count[g]) == len(res[g])
         assert [int(x) for x in got.ids[g * R:g * R + len(res[g])]] == [i for i, _ in res[g]]
+
+
+@pytest.mark.parametrize("admit_rule,objective", [(1, 0), (0, 1), (0, 2), (1, 1), (1, 2)])
+def test_placement_variants_against_brute_force(oracle, admit_rule, objective):
+    """Section 3.4: other objectives, and admission by the largest member drop (the comment in
+    Algorithm 2), against the exact-rational restatement."""
+    rng = np.random.default_rng(100 + 10 * admit_rule + objective)
+    P, G, R, n = 6, 5, 3, 80
+    Pm = (rng.integers(0, 40, (P, P)) / 64.0).astype(np.float32)
+    count = rng.integers(0, R, G)
+    ids = np.full(G * R, -1)
+    expiry = np.zeros(G * R, dtype=np.int64)
+    for g in range(G):
+        for s in range(count[g]):
+            ids[g * R + s] = rng.integers(0, P)
+            expiry[g * R + s] = rng.choice([0, 4, 9])
+    arr_id = rng.integers(0, P, n)
+    arr_life = rng.choice([0, 2, 5, 11], n)
+    want, _ = brute_place(Pm, G, R, ids, expiry, count, arr_id, arr_life, 0.5, admit_rule, objective)
+    got = oracle.place(Pm, G, R, ids, expiry, count, 0, arr_id, arr_life, 0.5, admit_rule, objective)
+    assert list(got.gpu) == want
+    base = oracle.place(Pm, G, R, ids, expiry, count, 0, arr_id, arr_life, 0.5)
+    assert list(base.gpu) != want          # the variant really decides differently on this stream
+
+
+def test_placement_variant_hand_cases(oracle):
+    # model 0 suffers 0.9 from model 1, model 1 nothing: mean 0.45 < 0.5 admits, largest drop 0.9 does not
+    Pm = np.array([[0, 0.9], [0.0, 0]], dtype=np.float32)
+    z = np.zeros(2)
+    assert list(oracle.place(Pm, 1, 2, [0, -1], z, [1], 0, [1], [0], 0.5, 0, 0).gpu) == [0]
+    assert list(oracle.place(Pm, 1, 2, [0, -1], z, [1], 0, [1], [0], 0.5, 1, 0).gpu) == [-1]
+    # two GPUs: g0 holds model 0 (arrival 1 hurts it by 0.3, suffers 0), g1 holds model 2 (arrival suffers 0.2,
+    # hurts by 0.05): mean 0.15 vs 0.125 -> g1; arrival's own drop 0 vs 0.2 -> g0; largest 0.3 vs 0.2 -> g1
+    Pm = np.zeros((3, 3), dtype=np.float32)
+    Pm[0, 1], Pm[1, 2], Pm[2, 1] = 0.3, 0.2, 0.05
+    args = (Pm, 2, 2, [0, -1, 2, -1], np.zeros(4), [1, 1], 0, [1], [0], 0.5)
+    assert list(oracle.place(*args, 0, 0).gpu) == [1]
+    assert list(oracle.place(*args, 0, 2).gpu) == [0]
+    assert list(oracle.place(*args, 0, 1).gpu) == [1]
 
 
 def test_placement_rules(oracle):
