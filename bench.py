@@ -282,6 +282,22 @@ def main():
     st0 = rm.ClusterState(G, R, cl.ids, cl.expiry, cl.count, 0)
     phase("placement_ms", lambda: rm.place(Pm, st0, darr[0], darr[1], cl.lam, want_mean=False))
 
+    # the same cluster shape as many independent arrival streams (one CTA each): what the GPU is for on
+    # this row, since a single stream is one dependent chain
+    S, nb = 8 * 148, min(2048, len(cl.arr_id))
+    roll = (np.arange(S)[:, None] * 7 + np.arange(nb)[None, :]) % len(cl.arr_id)
+    b_ids = torch.from_numpy(np.tile(cl.ids, (S, 1))).to(dev)
+    b_exp = torch.from_numpy(np.tile(cl.expiry.view(np.int32), (S, 1))).to(dev)
+    b_cnt = torch.from_numpy(np.tile(cl.count.view(np.int32), (S, 1))).to(dev)
+    b_aid = torch.from_numpy(cl.arr_id[roll]).to(dev)
+    b_life = torch.from_numpy(cl.arr_life.view(np.int32)[roll]).to(dev)
+
+    def batch_place():
+        rm.place_batch(Pm, G, R, b_ids.clone(), b_exp.clone(), b_cnt.clone(),
+                       torch.zeros(S, dtype=torch.int32, device=dev), b_aid, b_life, cl.lam)
+    batch_place()
+    phase("placement_batch_ms", batch_place)
+
     for _ in range(2):
         step_e2e()
     ms_e2e = timed(step_e2e, args.steps)
@@ -312,6 +328,8 @@ def main():
                        "placement": f"{G} gpus x {R} slots, {len(cl.arr_id)} arrivals",
                        "l2": "256 MB written between timed steps (L2 flush); the 24 MB library is re-read from L2 within a step"},
             "placements_per_s": len(cl.arr_id) / (phases["placement_ms"] * 1e-3),
+            "placements_per_s_batched": {"value": S * nb / (phases["placement_batch_ms"] * 1e-3), "streams": S,
+                                         "arrivals_per_stream": nb},
             "phases": phases,
             "e2e": {"value": evals_all * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": int(h2d_bytes), "d2h_bytes_per_step": int(P * P * 4 + 4 * len(cl.arr_id)),

@@ -136,7 +136,19 @@ typedef struct roomie_opts {
     int32_t start_filter;   /* 1: keep only alignments whose two start kernels interfere (Eq. 2) */
     float lambda;           /* degradation budget of Algorithm 2 (the paper uses 0.5)            */
     uint32_t max_residents; /* slots per GPU in the cluster state                                */
+    int32_t admit_rule;     /* ROOMIE_ADMIT_*: which quantity must stay below lambda             */
+    int32_t objective;      /* ROOMIE_OBJECTIVE_*: which quantity the chosen GPU minimises       */
 } roomie_opts;
+/* Algorithm 2 as printed admits a GPU when the MEAN drop of its would-be model set is below lambda
+ * and picks the lowest mean.  Its comment asks that "no variant has a performance drop beyond
+ * lambda" (ADMIT_MAX: the largest member drop), and Section 3.4 notes that the objective can be
+ * substituted: OBJECTIVE_MAX picks the GPU whose worst-hit member suffers least, OBJECTIVE_ARRIVAL
+ * the GPU on which the arriving model itself suffers least.  Ties go to the lowest GPU index. */
+#define ROOMIE_ADMIT_MEAN 0
+#define ROOMIE_ADMIT_MAX 1
+#define ROOMIE_OBJECTIVE_MEAN 0
+#define ROOMIE_OBJECTIVE_MAX 1
+#define ROOMIE_OBJECTIVE_ARRIVAL 2
 
 /* Unordered profile pairs (a <= b, diagonal included) are numbered row-major over the upper
  * triangle: (0,0), (0,1), ..., (0,P-1), (1,1), ...; there are P(P+1)/2 of them. */
@@ -238,11 +250,23 @@ typedef struct roomie_cluster_state {
  *   arr_id [n] profile ids, arr_life [n] lifetimes in arrival ticks;
  *   gpu_out [n]; mean_out [n] (optional) mean drop of the chosen GPU; mu_arr_out [n]
  *   (optional) predicted drop of the arriving model there.
- * Decisions are taken in float32 with the fixed summation order of roomie_multi_estimate.
+ * Decisions are taken in float32 with the fixed summation order of roomie_multi_estimate;
+ * opts->admit_rule and opts->objective select the variants described at roomie_opts.
  * Errors: INVALID_ARG, CUDA. */
 int roomie_place(const float *Pmat, uint32_t P, const roomie_cluster_state *state /* host struct */,
                  const int32_t *arr_id, const uint32_t *arr_life, uint32_t n, const roomie_opts *opts /* host */,
                  int32_t *gpu_out, float *mean_out, float *mu_arr_out, void *stream);
+
+/* roomie_place for num_streams INDEPENDENT arrival streams at once (what-if scenarios, one
+ * cluster per tenant, placement-quality studies): one CTA per stream, so streams run side by
+ * side where a single stream is a dependent chain.  Every per-stream array is the single-stream
+ * array repeated num_streams times, stream-major: states->ids and ->expiry [S][G*R], ->count
+ * [S][G], ->tick [S]; arr_id, arr_life and the outputs [S][n].  All streams share Pmat, the
+ * cluster shape, n and the options.  Same decisions as num_streams calls of roomie_place. */
+int roomie_place_batch(const float *Pmat, uint32_t P, const roomie_cluster_state *states /* host struct */,
+                       const int32_t *arr_id, const uint32_t *arr_life, uint32_t n, uint32_t num_streams,
+                       const roomie_opts *opts /* host */, int32_t *gpu_out, float *mean_out, float *mu_arr_out,
+                       void *stream);
 
 /* Text of a roomie_status; the last CUDA error code/text seen by this thread's calls. */
 const char *roomie_strerror(int status);

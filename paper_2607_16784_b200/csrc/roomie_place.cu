@@ -68,9 +68,29 @@ struct PlaceArgs {
     int matrix_mode;        // 0: whole matrix in shared memory, 1: row/column ring, 2: global loads
     int pair_cache;         // 1: resident-resident terms cached in shared memory ([R][R][G] floats)
     uint32_t gpus_per_warp; // fast kernel: GPUs owned by each warp
+    int admit_rule;         // 0: mean drop < lambda, 1: largest member drop < lambda
+    int objective;          // 0: lowest mean drop, 1: lowest largest drop, 2: lowest drop of the arrival
 };
 
 constexpr unsigned long long kNoGpu = ~0ull;
+
+// one CTA per independent arrival stream: stream s owns slice s of every per-stream array
+__device__ __forceinline__ void select_stream(PlaceArgs& g) {
+    const size_t s = blockIdx.x;
+    g.ids += s * g.G * g.R; g.expiry += s * g.G * g.R; g.count += s * g.G; g.tick += s;
+    g.arr_id += s * g.n; g.arr_life += s * g.n; g.gpu_out += s * g.n;
+    if (g.mean_out) g.mean_out += s * g.n;
+    if (g.mu_arr_out) g.mu_arr_out += s * g.n;
+}
+
+// Algorithm 2 line 7 and the choice criterion (Section 3.4 allows other objectives): returns the bits
+// of the score to minimise, or all ones when the GPU is not admissible.  All quantities are >= 0, so
+// their float bits order like the floats.
+__device__ __forceinline__ uint32_t decision_key(const PlaceArgs& g, float mean, float worst, float mu_inc) {
+    const float admit = g.admit_rule == 1 ? worst : mean;
+    const float score = g.objective == 1 ? worst : g.objective == 2 ? mu_inc : mean;
+    return admit < g.lambda ? __float_as_uint(score) : 0xffffffffu;
+}
 constexpr uint32_t kArrChunk = 1024;      // arrivals staged in shared memory at a time
 constexpr int kRing = 4;      // arrival k+2 is fetched while k is scored and k-1's winner still reads its column
 
@@ -86,6 +106,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // kSlots = 0: plain loops for any R
 template <int kSlots>
 __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
+    select_stream(g);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t G = g.G, R = g.R, P = g.P, GR = G * R;
     int32_t* s_ids = reinterpret_cast<int32_t*>(smem_raw);
@@ -205,7 +226,7 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
                     recompute_partials(c);
                 }
                 if (c < R) {                                           // what-if: residents + the arrival
-                    float tot = 0.0f;
+                    float tot = 0.0f, worst = 0.0f;
                     if constexpr (kSlots > 0) {
                         float to_inc[kSlots], from_inc[kSlots], part[kSlots];
 #pragma unroll
@@ -220,21 +241,25 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
 #pragma unroll
                         for (int t = 0; t < kSlots; ++t) {
                             if ((uint32_t)t < c) {
-                                tot = __fadd_rn(tot, __fadd_rn(part[t], to_inc[t]));
+                                const float mu_t = __fadd_rn(part[t], to_inc[t]);
+                                worst = fmaxf(worst, mu_t);
+                                tot = __fadd_rn(tot, mu_t);
                                 mu_inc = __fadd_rn(mu_inc, from_inc[t]);
                             }
                         }
                     } else {
                         for (uint32_t t = 0; t < c; ++t) {
                             const int32_t id = ID(t);
-                            tot = __fadd_rn(tot, __fadd_rn(PA(t), col_inc[(size_t)id * col_stride]));
+                            const float mu_t = __fadd_rn(PA(t), col_inc[(size_t)id * col_stride]);
+                            worst = fmaxf(worst, mu_t);
+                            tot = __fadd_rn(tot, mu_t);
                             mu_inc = __fadd_rn(mu_inc, row_inc[id]);
                         }
                     }
                     tot = __fadd_rn(tot, mu_inc);
                     mean = __fdiv_rn(tot, (float)(c + 1));
-                    if (mean < g.lambda)                               // Algorithm 2 line 7
-                        key = ((unsigned long long)__float_as_uint(mean) << 32) | tid;
+                    const uint32_t kb = decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
+                    if (kb != 0xffffffffu) key = ((unsigned long long)kb << 32) | tid;
                 }
             }
             // argmin over GPUs, lowest index on equal means (mean >= 0, so its bits order as integers)
@@ -314,6 +339,7 @@ __device__ __forceinline__ void cp_async_4_s(uint32_t smem_addr, const void* gme
 }
 
 __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
+    select_stream(g);
     // one float/int array; every region is addressed by a 32-bit word index
     extern __shared__ __align__(16) float sm[];
     int32_t* smi = reinterpret_cast<int32_t*>(sm);
@@ -448,7 +474,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             uint32_t key_hi = 0xffffffffu;
             float mean = 0.0f, mu_inc = 0.0f;
             if (owner && c < R) {                                            // what-if: residents + the arrival
-                float tot = 0.0f;
+                float tot = 0.0f, worst = 0.0f;
                 for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {
                     const uint32_t p = o & 15u;
                     const uint32_t d1 = (uint32_t)((int32_t)kg - smi[oBI + p * G]);   // arrivals since placed, minus 1 (huge if old)
@@ -456,12 +482,14 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                     const uint32_t i0 = young ? young_k + 2 * d1 : ring_k + p * G;
                     const float to = sm[i0];                                  // P[id][inc]
                     const float from = sm[i0 + (young ? 1u : GR)];            // P[inc][id]
-                    tot = __fadd_rn(tot, __fadd_rn(sm[oPA + p * G], to));
+                    const float mu_t = __fadd_rn(sm[oPA + p * G], to);
+                    worst = fmaxf(worst, mu_t);
+                    tot = __fadd_rn(tot, mu_t);
                     mu_inc = __fadd_rn(mu_inc, from);
                 }
                 tot = __fadd_rn(tot, mu_inc);
                 mean = __fdiv_rn(tot, (float)(c + 1));
-                if (mean < g.lambda) key_hi = __float_as_uint(mean);         // Algorithm 2 line 7; mean >= 0: bits order
+                key_hi = decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
             }
             const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
             const uint32_t best_lo = __reduce_min_sync(0xffffffffu, (key_hi == best_hi && key_hi != 0xffffffffu) ? gpu : 0xffffffffu);
@@ -542,17 +570,20 @@ extern "C" int roomie_multi_estimate(const float* Pmat, uint32_t P, const int32_
     return ROOMIE_OK;
 }
 
-extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_state* state, const int32_t* arr_id,
-                            const uint32_t* arr_life, uint32_t n, const roomie_opts* opts, int32_t* gpu_out,
-                            float* mean_out, float* mu_arr_out, void* stream) {
+static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state* state, const int32_t* arr_id,
+                      const uint32_t* arr_life, uint32_t n, uint32_t num_streams, const roomie_opts* opts,
+                      int32_t* gpu_out, float* mean_out, float* mu_arr_out, void* stream) {
     if (!Pmat || P == 0 || !state || !opts || !state->ids || !state->expiry || !state->count || !state->tick)
         return ROOMIE_ERR_INVALID_ARG;
     if (state->num_gpus == 0 || state->num_gpus > 1024 || state->max_residents == 0 || state->max_residents > 64 ||
         (uint64_t)state->num_gpus * state->max_residents > 8192)
         return ROOMIE_ERR_INVALID_ARG;
-    if (n == 0) return ROOMIE_OK;
+    if (n == 0 || num_streams == 0) return ROOMIE_OK;
     if (!arr_id || !arr_life || !gpu_out) return ROOMIE_ERR_INVALID_ARG;
+    if (opts->admit_rule < 0 || opts->admit_rule > 1 || opts->objective < 0 || opts->objective > 2)
+        return ROOMIE_ERR_INVALID_ARG;
     PlaceArgs a;
+    a.admit_rule = opts->admit_rule; a.objective = opts->objective;
     a.Pm = Pmat; a.P = P; a.G = state->num_gpus; a.R = state->max_residents;
     a.ids = state->ids; a.expiry = state->expiry; a.count = state->count; a.tick = state->tick;
     a.arr_id = arr_id; a.arr_life = arr_life; a.n = n; a.lambda = opts->lambda;
@@ -569,7 +600,7 @@ extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_
         auto kern = place_fast_kernel;
         if (fast_bytes > 48 * 1024)
             ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast_bytes));
-        kern<<<1, threads, fast_bytes, st>>>(a);
+        kern<<<num_streams, threads, fast_bytes, st>>>(a);
         note_launch();
         ROOMIE_CUDA_OK(cudaGetLastError());
         return ROOMIE_OK;
@@ -589,8 +620,21 @@ extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_
     auto kern = a.R <= 16 ? place_kernel<16> : place_kernel<0>;
     if (smem > 48 * 1024)
         ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<1, threads, smem, st>>>(a);
+    kern<<<num_streams, threads, smem, st>>>(a);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;
+}
+
+extern "C" int roomie_place(const float* Pmat, uint32_t P, const roomie_cluster_state* state, const int32_t* arr_id,
+                            const uint32_t* arr_life, uint32_t n, const roomie_opts* opts, int32_t* gpu_out,
+                            float* mean_out, float* mu_arr_out, void* stream) {
+    return place_impl(Pmat, P, state, arr_id, arr_life, n, 1, opts, gpu_out, mean_out, mu_arr_out, stream);
+}
+
+extern "C" int roomie_place_batch(const float* Pmat, uint32_t P, const roomie_cluster_state* states,
+                                  const int32_t* arr_id, const uint32_t* arr_life, uint32_t n, uint32_t num_streams,
+                                  const roomie_opts* opts, int32_t* gpu_out, float* mean_out, float* mu_arr_out,
+                                  void* stream) {
+    return place_impl(Pmat, P, states, arr_id, arr_life, n, num_streams, opts, gpu_out, mean_out, mu_arr_out, stream);
 }

@@ -17,7 +17,7 @@ EXPORTS = [
     "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
     "roomie_pair_interference_static",
-    "roomie_multi_estimate", "roomie_place", "roomie_strerror", "roomie_last_cuda_error",
+    "roomie_multi_estimate", "roomie_place", "roomie_place_batch", "roomie_strerror", "roomie_last_cuda_error",
     "roomie_launch_count", "roomie_reset_launch_count", "roomie_profile_enable", "roomie_profile_walk_ms",
 ]
 
@@ -54,6 +54,8 @@ def _load():
                                           C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p]
     dll.roomie_place.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32,
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    dll.roomie_place_batch.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32,
+                                       C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     return dll
 
 
@@ -91,7 +93,8 @@ class _Library(C.Structure):
 
 class _Opts(C.Structure):
     _fields_ = [("walk_mode", C.c_int32), ("n_align", C.c_uint32), ("start_filter", C.c_int32),
-                ("lam", C.c_float), ("max_residents", C.c_uint32)]
+                ("lam", C.c_float), ("max_residents", C.c_uint32), ("admit_rule", C.c_int32),
+                ("objective", C.c_int32)]
 
 
 class _Detail(C.Structure):
@@ -211,8 +214,9 @@ def library_build(grid, threads, regs, smem, dur_us, gap_us, offsets, spec, stre
     return lib
 
 
-def _opts(mode=TIMELINE, n_align=1, start_filter=0, lam=0.5, max_residents=0) -> _Opts:
-    return _Opts(int(mode), int(n_align), int(start_filter), float(lam), int(max_residents))
+def _opts(mode=TIMELINE, n_align=1, start_filter=0, lam=0.5, max_residents=0, admit_rule=0, objective=0) -> _Opts:
+    return _Opts(int(mode), int(n_align), int(start_filter), float(lam), int(max_residents),
+                 int(admit_rule), int(objective))
 
 
 def pair_workspace_bytes(lib: Library, *, mode=TIMELINE, n_align=1, start_filter=0,
@@ -339,7 +343,8 @@ class ClusterState:
         return self
 
 
-def place(Pmat, state: ClusterState, arr_id, arr_life, lam=0.5, want_mean=True, stream=None):
+def place(Pmat, state: ClusterState, arr_id, arr_life, lam=0.5, want_mean=True, stream=None,
+          admit_rule=0, objective=0):
     """roomie_place: Algorithm 2 over a stream of arrivals.  Returns (gpu int32 [n], mean, mu_arr)."""
     Pm = _dev(Pmat, torch.float32)
     aid = _dev(arr_id, torch.int32)
@@ -349,10 +354,35 @@ def place(Pmat, state: ClusterState, arr_id, arr_life, lam=0.5, want_mean=True, 
     gpu = torch.empty(n, dtype=torch.int32, device=Pm.device)
     mean = torch.empty(n, dtype=torch.float32, device=Pm.device) if want_mean else None
     mu_arr = torch.empty(n, dtype=torch.float32, device=Pm.device) if want_mean else None
-    o = _opts(lam=lam, max_residents=state.max_residents)
+    o = _opts(lam=lam, max_residents=state.max_residents, admit_rule=admit_rule, objective=objective)
     _check(_dll.roomie_place(_ptr(Pm), Pm.shape[0], C.byref(state.c), _ptr(aid), _ptr(life), n, C.byref(o),
                              _ptr(gpu), _ptr(mean), _ptr(mu_arr), _stream(stream)), "roomie_place")
     return gpu, mean, mu_arr
+
+
+def place_batch(Pmat, num_gpus, max_residents, ids, expiry, count, tick, arr_id, arr_life, lam=0.5,
+                want_mean=False, stream=None, admit_rule=0, objective=0):
+    """roomie_place_batch: S independent arrival streams, one CTA each.  ids/expiry [S, G*R], count [S, G],
+    tick [S], arr_id/arr_life [S, n] (int32 device tensors or arrays; the state tensors are updated in place
+    when they already are contiguous int32 device tensors).  Returns (gpu int32 [S, n], mean, mu_arr, state)."""
+    Pm = _dev(Pmat, torch.float32)
+    u32 = lambda x: x if isinstance(x, torch.Tensor) else np.asarray(x, dtype=np.uint32).view(np.int32)
+    ids_t, exp_t, cnt_t, tick_t = (_dev(ids, torch.int32), _dev(u32(expiry), torch.int32),
+                                   _dev(u32(count), torch.int32), _dev(u32(tick), torch.int32))
+    aid, life = _dev(arr_id, torch.int32), _dev(u32(arr_life), torch.int32)
+    S, n = aid.shape[0], aid.shape[1]
+    if ids_t.numel() != S * num_gpus * max_residents or cnt_t.numel() != S * num_gpus or tick_t.numel() != S \
+            or life.shape != aid.shape:
+        raise ValueError("per-stream arrays do not match the number of streams")
+    state = _State(int(num_gpus), int(max_residents), ids_t.data_ptr(), exp_t.data_ptr(), cnt_t.data_ptr(),
+                   tick_t.data_ptr())
+    gpu = torch.empty((S, n), dtype=torch.int32, device=Pm.device)
+    mean = torch.empty((S, n), dtype=torch.float32, device=Pm.device) if want_mean else None
+    mu_arr = torch.empty((S, n), dtype=torch.float32, device=Pm.device) if want_mean else None
+    o = _opts(lam=lam, max_residents=max_residents, admit_rule=admit_rule, objective=objective)
+    _check(_dll.roomie_place_batch(_ptr(Pm), Pm.shape[0], C.byref(state), _ptr(aid), _ptr(life), n, S, C.byref(o),
+                                   _ptr(gpu), _ptr(mean), _ptr(mu_arr), _stream(stream)), "roomie_place_batch")
+    return gpu, mean, mu_arr, dict(ids=ids_t, expiry=exp_t, count=cnt_t, tick=tick_t)
 
 
 def launch_count() -> int:

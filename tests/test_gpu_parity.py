@@ -355,3 +355,61 @@ def test_placement_edge_cases(rm, oracle):
     gpu = rm.place(huge, st, cl.arr_id, cl.arr_life, 0.5)[0].cpu().numpy()
     want = oracle.place(huge, cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0, cl.arr_id, cl.arr_life, 0.5)
     assert np.array_equal(gpu, want.gpu)
+
+
+# ----------------------------------------------------------------------------- placement variants, batches
+@pytest.mark.parametrize("cfg", [2, 4])
+@pytest.mark.parametrize("admit_rule,objective", [(1, 0), (0, 1), (0, 2), (1, 2)])
+def test_placement_variants_bit_exact(rm, oracle, cfg, admit_rule, objective):
+    """Admission by the largest member drop and the alternative objectives (Section 3.4), same matrix on
+    both sides: every decision identical."""
+    lib = rs.make_library(cfg)
+    cl = rs.make_cluster(cfg)
+    _, gl = build_both(rm, oracle, lib)
+    Pm32 = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)[0].cpu().numpy()
+    st = rm.ClusterState(cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0)
+    gpu, mean, mu_arr = rm.place(Pm32, st, cl.arr_id, cl.arr_life, cl.lam, admit_rule=admit_rule, objective=objective)
+    want = oracle.place(Pm32, cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0,
+                        cl.arr_id, cl.arr_life, cl.lam, admit_rule, objective)
+    assert np.array_equal(gpu.cpu().numpy(), want.gpu)
+    assert np.array_equal(mean.cpu().numpy().view(np.uint32), want.mean.view(np.uint32))
+    assert np.array_equal(st.ids.cpu().numpy(), want.ids)
+
+
+def test_placement_variants_generic_kernel(rm, oracle):
+    """More than 8 slots per GPU takes the generic kernel: same rules there."""
+    rng = np.random.default_rng(9)
+    P, G, R, n = 40, 6, 12, 400
+    Pm = (rng.random((P, P)) * 0.2).astype(np.float32)
+    aid = rng.integers(0, P, n).astype(np.int32)
+    life = rng.integers(1, 60, n).astype(np.uint32)
+    for admit_rule, objective in ((0, 0), (1, 0), (0, 1), (1, 2)):
+        st = rm.ClusterState(G, R, [-1] * (G * R), [0] * (G * R), [0] * G, 3)
+        gpu = rm.place(Pm, st, aid, life, 0.5, admit_rule=admit_rule, objective=objective)[0].cpu().numpy()
+        want = oracle.place(Pm, G, R, [-1] * (G * R), [0] * (G * R), [0] * G, 3, aid, life, 0.5, admit_rule, objective)
+        assert np.array_equal(gpu, want.gpu) and np.array_equal(st.ids.cpu().numpy(), want.ids)
+
+
+@pytest.mark.parametrize("shape", [(64, 8), (8, 4), (5, 12)])
+def test_place_batch_equals_single_streams(rm, oracle, shape):
+    """Independent streams side by side (one CTA each) decide exactly like one stream at a time."""
+    G, R = shape
+    S, n, P = 37, 300, 32
+    lib = rs.make_library(2)
+    _, gl = build_both(rm, oracle, lib)
+    Pm32 = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)[0].cpu().numpy()
+    ids = np.full((S, G * R), -1, np.int32); exp = np.zeros((S, G * R), np.uint32)
+    cnt = np.zeros((S, G), np.uint32); tick = np.arange(S, dtype=np.uint32) * 5
+    aid = np.zeros((S, n), np.int32); life = np.zeros((S, n), np.uint32)
+    for s in range(S):
+        cl = rs.make_cluster(2, seed=1000 + s, num_profiles=P, num_gpus=G, max_residents=R, num_arrivals=n)
+        ids[s], exp[s], cnt[s], aid[s], life[s] = cl.ids, cl.expiry, cl.count, cl.arr_id, cl.arr_life
+    gpu, mean, mu_arr, state = rm.place_batch(Pm32, G, R, ids, exp, cnt, tick, aid, life, 0.5, want_mean=True)
+    gpu, mean = gpu.cpu().numpy(), mean.cpu().numpy()
+    for s in range(S):
+        want = oracle.place(Pm32, G, R, ids[s], exp[s], cnt[s], int(tick[s]), aid[s], life[s], 0.5)
+        assert np.array_equal(gpu[s], want.gpu), s
+        assert np.array_equal(mean[s].view(np.uint32), want.mean.view(np.uint32))
+        assert np.array_equal(state["ids"].cpu().numpy().reshape(S, -1)[s], want.ids)
+        assert np.array_equal(state["count"].cpu().numpy().view(np.uint32).reshape(S, -1)[s], want.count)
+        assert int(state["tick"].cpu().numpy().view(np.uint32)[s]) == want.tick
