@@ -54,8 +54,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="roomie", choices=["roomie", "reference"])
     ap.add_argument("--config", type=int, default=3, help="library configuration (0-4)")
-    ap.add_argument("--setting", default="base", choices=["base", "greedy"],
-                    help="base: alignment (0,0); greedy: 8x8 alignments, start filter, median")
+    ap.add_argument("--setting", default="base", choices=["base", "greedy", "lockstep_full"],
+                    help="base: alignment (0,0); greedy: 8x8 alignments, start filter, median; lockstep_full: "
+                         "Algorithm 1 as printed over the full Cartesian alignment set (use configs 1, 2 or 4)")
     ap.add_argument("--arrivals", type=int, default=10000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profiles", type=int, default=None, help="truncate the library (ncu captures)")
@@ -64,7 +65,16 @@ def parse_args():
 
 
 def setting_kw(name):
+    if name == "lockstep_full":
+        return dict(mode=1, n_align=0, start_filter=1)
     return dict(mode=0, n_align=1, start_filter=0) if name == "base" else dict(mode=0, n_align=8, start_filter=1)
+
+
+def oracle_sample_pairs(setting, total_pairs):
+    """Pairs the CPU oracle is timed on: all of them at the base setting, a bounded prefix otherwise."""
+    if setting == "base":
+        return total_pairs
+    return max(1, total_pairs // (32 if setting == "greedy" else 512))
 
 
 def make_inputs(cfg, rank, num_profiles, arrivals):
@@ -142,7 +152,7 @@ def run_reference(args, rank, world):
     P = lib.num_profiles
     total_pairs = P * (P + 1) // 2
     # bounded sample: the base setting runs whole; the greedy one on the first 1/32 of the pairs
-    pair_end = total_pairs if args.setting == "base" else max(1, total_pairs // 32)
+    pair_end = oracle_sample_pairs(args.setting, total_pairs)
     sample = ("full workload" if pair_end == total_pairs else f"first {pair_end} of {total_pairs} pairs") + \
              f", {len(cl.arr_id)} arrivals"
     for _ in range(min(args.warmup, 1)):
@@ -319,6 +329,21 @@ def main():
         per_launch_ms = walk_ms / max(walk_launches, 1)
         launches_per_matrix = walk_launches / args.steps
         achieved = alg / launches_per_matrix / (per_launch_ms * 1e-3) / 1e9 if walk_launches else None
+        if args.setting == "lockstep_full":
+            # compute-bound kernel: table cells visited (q_a*q_b per pair, at most 4 passes of the exact
+            # median) against the plain-ALU issue peak, 148 SMs x 128 lanes x SM clock, divided by the 54
+            # lane-instructions one cell visit takes (profiles/lockstep_full_kernel_config2.md)
+            q = lib.q().astype(np.int64)
+            ia, ib = np.triu_indices(P)
+            visits = 4.0 * float((q[ia] * q[ib]).sum())
+            peak_visits = 148 * 128 * 1.965e9 / 54.0 / 1e9
+            ach = visits / (per_launch_ms * 1e-3) / 1e9 if walk_launches else None
+            roofline = {"bound": "alu", "kernel": "lockstep_full_kernel", "achieved": ach, "peak": peak_visits,
+                        "unit": "G cell visits/s", "frac": (ach / peak_visits) if ach else None,
+                        "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz / 54 lane-instructions per visit",
+                        "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix, "traffic": None}
+        else:
+            roofline = None
         line = {
             "metric": METRIC, "value": evals_all * args.steps / (ms_dev * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_dev / args.steps,
@@ -336,7 +361,7 @@ def main():
                     "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "timeline_tiles_kernel", "achieved": achieved, "peak": peak,
+            "roofline": roofline or {"bound": "hbm", "kernel": "lockstep_full_kernel" if args.setting == "lockstep_full" else "timeline_tiles_kernel", "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": alg / launches_per_matrix if walk_launches else None,
                          "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix,
@@ -348,7 +373,7 @@ def main():
             import oracle
             oracle.build()
             total_pairs = P * (P + 1) // 2
-            pair_end = total_pairs if args.setting == "base" else max(1, total_pairs // 32)
+            pair_end = oracle_sample_pairs(args.setting, total_pairs)
             s, ev, _ = oracle_step(oracle, lib, cl, kw, pair_end, args.oracle_threads)
             line["cpu_baseline"] = {"value": ev / s, "unit": UNIT, "cores": args.oracle_threads or oracle.max_threads(), "kind": "oracle",
                                     "sample": ("full workload" if pair_end == total_pairs else

@@ -131,8 +131,13 @@ int roomie_library_build(const roomie_library *lib /* host */, const roomie_kern
                                   duration d_k is charged                                        */
 typedef struct roomie_opts {
     int32_t walk_mode;      /* ROOMIE_WALK_*                                                      */
-    uint32_t n_align;       /* A: alignment set = A x A evenly spaced start indices
-                               floor(t*q/A); 0 = the full Cartesian product (small profiles only) */
+    uint32_t n_align;       /* A: alignment set = A x A evenly spaced start indices floor(t*q/A);
+                               0 = the full Cartesian product q_i x q_j.  With ROOMIE_WALK_LOCKSTEP
+                               that is Algorithm 1 exactly as printed and is served for any profile
+                               length (all alignments of a pair are suffix sums along the diagonals
+                               of one q_i x q_j table, exact median by radix select); with
+                               ROOMIE_WALK_TIMELINE, or when per-alignment detail is requested,
+                               at most 4096 alignments per pair                                  */
     int32_t start_filter;   /* 1: keep only alignments whose two start kernels interfere (Eq. 2) */
     float lambda;           /* degradation budget of Algorithm 2 (the paper uses 0.5)            */
     uint32_t max_residents; /* slots per GPU in the cluster state                                */

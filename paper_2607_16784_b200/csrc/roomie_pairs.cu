@@ -427,19 +427,23 @@ __device__ float select_rank(const float* v, uint32_t n, uint32_t k, int lane) {
 }
 
 // P[a][b], P[b][a] from the two medians (gamma = max(q_i/q_j, 1), Eq. 4 with M = {i, j})
-__device__ __forceinline__ void store_pair(const FinalArgs& g, uint32_t a, uint32_t b, uint32_t qa, uint32_t qb,
-                                           float med_i, float med_j) {
-    const unsigned long long Ta = g.lib.T[a], Tb = g.lib.T[b];
+__device__ __forceinline__ void store_pair_values(const LibView& lib, const PairSet& ps, float* P_out, uint32_t a,
+                                                  uint32_t b, uint32_t qa, uint32_t qb, float med_i, float med_j) {
+    const unsigned long long Ta = lib.T[a], Tb = lib.T[b];
     const float fa = (float)qa, fb = (float)qb;
     const float g_ab = fmaxf(__fdiv_rn(fa, fb), 1.0f), g_ba = fmaxf(__fdiv_rn(fb, fa), 1.0f);
     const float p_ab = Ta ? __fdiv_rn(g_ab * med_i, (float)Ta) : 0.0f;
     const float p_ba = Tb ? __fdiv_rn(g_ba * med_j, (float)Tb) : 0.0f;
-    if (g.ps.explicit_pair) {
-        g.P_out[0] = p_ab; g.P_out[1] = p_ba;
+    if (ps.explicit_pair) {
+        P_out[0] = p_ab; P_out[1] = p_ba;
     } else {
-        g.P_out[(size_t)a * g.lib.P + b] = p_ab;
-        if (a != b) g.P_out[(size_t)b * g.lib.P + a] = p_ba;
+        P_out[(size_t)a * lib.P + b] = p_ab;
+        if (a != b) P_out[(size_t)b * lib.P + a] = p_ba;
     }
+}
+__device__ __forceinline__ void store_pair(const FinalArgs& g, uint32_t a, uint32_t b, uint32_t qa, uint32_t qb,
+                                           float med_i, float med_j) {
+    store_pair_values(g.lib, g.ps, g.P_out, a, b, qa, qb, med_i, med_j);
 }
 
 // one warp per pair: ordered sum of the tile partials of every alignment, ordered compaction of
@@ -540,6 +544,8 @@ __global__ void __launch_bounds__(256) finalize_single_kernel(FinalArgs g) {
     if ((threadIdx.x & 31) == 0 && g.evals_out && evals) atomicAdd(g.evals_out, evals);
 }
 
+#include "roomie_lockstep_full.cuh"
+
 // ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
@@ -611,6 +617,31 @@ static int slots_for(const roomie_library* lib, const roomie_opts* o, bool expli
     slots = (uint32_t)m;
     return ROOMIE_OK;
 }
+
+// Algorithm 1 as printed with the full Cartesian alignment set: no scratch, one CTA per pair
+static int run_lockstep_full(const roomie_library* lib, const roomie_opts* o, const PairSet& ps, float* P_out,
+                             uint64_t* evals_out, cudaStream_t st) {
+    FullArgs fa;
+    fa.lib.records = static_cast<const uint4*>(lib->records);
+    fa.lib.offsets = lib->offsets;
+    fa.lib.T = reinterpret_cast<const unsigned long long*>(lib->T);
+    fa.lib.P = lib->num_profiles;
+    fa.lib.cap = make_cap(lib->spec);
+    fa.ps = ps; fa.start_filter = o->start_filter;
+    fa.inv_table = lib->share_table;
+    fa.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u;
+    fa.P_out = P_out; fa.evals_out = reinterpret_cast<unsigned long long*>(evals_out);
+    uint32_t grid = (uint32_t)sm_count() * 3u;
+    if (grid > ps.n_pairs) grid = ps.n_pairs;
+    profile_mark(st, true);
+    lockstep_full_kernel<<<grid, kFullThreads, fa.n_inv * sizeof(float), st>>>(fa);
+    profile_mark(st, false);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+    return ROOMIE_OK;
+}
+
+static bool wants_lockstep_full(const roomie_opts* o) { return o->walk_mode == ROOMIE_WALK_LOCKSTEP && o->n_align == 0; }
 
 static int check_lib(const roomie_library* lib, const roomie_opts* o) {
     if (!lib || !o || !lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->share_table ||
@@ -728,6 +759,7 @@ extern "C" size_t roomie_pair_workspace_bytes(const roomie_library* lib, const r
     const uint64_t total = (uint64_t)lib->num_profiles * (lib->num_profiles + 1) / 2;
     if (pair_end > total) pair_end = total;
     if (pair_begin >= pair_end) return 0;
+    if (wants_lockstep_full(opts)) return 256;                       // that path keeps everything on chip
     uint32_t slots;
     if (slots_for(lib, opts, false, 0, 0, slots) != ROOMIE_OK) return 0;
     Need need;
@@ -747,6 +779,12 @@ extern "C" int roomie_pair_matrix(const roomie_library* lib, const roomie_opts* 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), st));
     if (pair_begin == pair_end) return ROOMIE_OK;
+    if (wants_lockstep_full(opts)) {
+        if (pair_end - pair_begin >= (1ull << 31)) return ROOMIE_ERR_CAPACITY;
+        PairSet ps;
+        ps.pair_begin = pair_begin; ps.n_pairs = (uint32_t)(pair_end - pair_begin); ps.explicit_pair = 0; ps.a = ps.b = 0;
+        return run_lockstep_full(lib, opts, ps, P_out, evals_out, st);
+    }
     uint32_t slots;
     rc = slots_for(lib, opts, false, 0, 0, slots);
     if (rc != ROOMIE_OK) return rc;
@@ -781,6 +819,11 @@ extern "C" int roomie_pair_interference(const roomie_library* lib, uint32_t a, u
         return ROOMIE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), st));
+    if (wants_lockstep_full(opts) && !detail) {
+        PairSet fps;
+        fps.pair_begin = 0; fps.n_pairs = 1; fps.explicit_pair = 1; fps.a = a; fps.b = b;
+        return run_lockstep_full(lib, opts, fps, out2, evals_out, st);
+    }
     uint32_t slots;
     rc = slots_for(lib, opts, true, a, b, slots);
     if (rc != ROOMIE_OK) return rc;
@@ -798,6 +841,13 @@ extern "C" int roomie_pair_interference_static(const roomie_library* lib, uint32
     int rc = check_lib(lib, opts);
     if (rc != ROOMIE_OK) return rc;
     if (!out2 || a >= lib->num_profiles || b >= lib->num_profiles) return ROOMIE_ERR_INVALID_ARG;
+    if (wants_lockstep_full(opts) && !detail) {                      // that path needs no scratch at all
+        cudaStream_t fst = static_cast<cudaStream_t>(stream);
+        if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), fst));
+        PairSet fps;
+        fps.pair_begin = 0; fps.n_pairs = 1; fps.explicit_pair = 1; fps.a = a; fps.b = b;
+        return run_lockstep_full(lib, opts, fps, out2, evals_out, fst);
+    }
     uint32_t slots;
     rc = slots_for(lib, opts, true, a, b, slots);
     if (rc != ROOMIE_OK) return rc;

@@ -413,3 +413,55 @@ def test_place_batch_equals_single_streams(rm, oracle, shape):
         assert np.array_equal(state["ids"].cpu().numpy().reshape(S, -1)[s], want.ids)
         assert np.array_equal(state["count"].cpu().numpy().view(np.uint32).reshape(S, -1)[s], want.count)
         assert int(state["tick"].cpu().numpy().view(np.uint32)[s]) == want.tick
+
+
+# ----------------------------------------------------------------------------- Algorithm 1 as printed, full alignment set
+@pytest.mark.parametrize("start_filter", [0, 1])
+def test_lockstep_full_cartesian_small_configs(rm, oracle, start_filter):
+    """Lock-step walk from every pair of start indices, exact median (configurations 0 and 1, every pair)."""
+    for cfg, feasible in ((0, True), (0, False), (1, True)):
+        lib = rs.make_library(cfg, feasible=feasible)
+        ol, gl = build_both(rm, oracle, lib)
+        want, want_ev = oracle.pair_matrix(ol, mode=1, n_align=0, start_filter=start_filter)
+        got, ev = rm.pair_matrix(gl, mode=1, n_align=0, start_filter=start_filter)
+        assert int(ev.item()) == want_ev
+        assert_close(got.cpu().numpy(), want)
+        assert gl.status_flags() == 0
+
+
+def test_lockstep_full_cartesian_long_profiles_and_special_cases(rm, oracle):
+    from test_oracle_walk import make_lib
+    lib = rs.make_library(2)
+    ol, gl = build_both(rm, oracle, lib)
+    q = lib.q()
+    order = np.argsort(q)
+    a, b = int(order[len(q) // 2]), int(order[len(q) // 2 + 1])          # two mid-sized profiles (~1000 kernels)
+    for sf in (0, 1):
+        for x, y in ((a, b), (b, a), (a, a)):
+            want = oracle.pair(ol, x, y, mode=1, n_align=0, start_filter=sf, cap_align=1)
+            got = rm.pair_interference(gl, x, y, mode=1, n_align=0, start_filter=sf)
+            assert int(got["evals"].item()) == want.evals
+            assert_close(got["P2"].cpu().numpy(), [want.P_ab, want.P_ba])
+            st = rm.pair_interference_static(gl, x, y, mode=1, n_align=0, start_filter=sf)
+            assert np.array_equal(st["P2"].cpu().numpy(), got["P2"].cpu().numpy())
+    # closed form: identical self-interfering kernels, delta(s_i, s_j) = D/2 * min(q - s_i, q - s_j)
+    k = (256, 64, 0, 10000, 0.05, 0.0)
+    for qa, qb in ((8, 8), (2, 2), (3, 1), (1, 1), (40, 17)):
+        lib2 = make_lib([[k] * qa, [k] * qb])
+        ol2 = oracle.library_build(lib2)
+        gl2 = rm.library_build(lib2.grid_blocks, lib2.block_threads, lib2.regs_per_thread, lib2.smem_per_block,
+                               lib2.dur_us, lib2.gap_us, lib2.offsets, lib2.spec)
+        vals = sorted(25000.0 * min(qa - i, qb - j) for i in range(qa) for j in range(qb))
+        med = 0.5 * (vals[(len(vals) - 1) // 2] + vals[len(vals) // 2])
+        got = rm.pair_interference(gl2, 0, 1, mode=1, n_align=0)["P2"].cpu().numpy()
+        assert got[0] == pytest.approx(max(qa / qb, 1.0) * med / (qa * 50000.0), rel=1e-6)
+        want = oracle.pair(ol2, 0, 1, mode=1, n_align=0, cap_align=1)
+        assert_close(got, [want.P_ab, want.P_ba])
+    # nothing interferes: kept set empty under the filter, all delays zero without it
+    small = (64, 16, 0, 100, 0.01, 0.001)
+    lib3 = make_lib([[small] * 30, [small] * 20])
+    gl3 = rm.library_build(lib3.grid_blocks, lib3.block_threads, lib3.regs_per_thread, lib3.smem_per_block,
+                           lib3.dur_us, lib3.gap_us, lib3.offsets, lib3.spec)
+    for sf in (0, 1):
+        r = rm.pair_interference(gl3, 0, 1, mode=1, n_align=0, start_filter=sf)
+        assert r["P2"].cpu().tolist() == [0.0, 0.0] and int(r["evals"].item()) == (0 if sf else sum(min(30 - i, 20 - j) for i in range(30) for j in range(20)))
