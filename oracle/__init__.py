@@ -243,3 +243,27 @@ def place(Pm32, num_gpus, max_residents, ids, expiry, count, tick, arr_id, arr_l
                         C.c_uint32(n), C.c_float(lam), C.c_int(admit_rule), C.c_int(objective),
                         _p(gpu), _p(mean), _p(mu_arr), _p(near))
     return Placement(gpu, mean, mu_arr, near, ids, expiry, count, int(t.value))
+
+
+def assignment_cost(Pm32, models, gpu_of):
+    """Average predicted drop of a deployment (float32 as defined, float64 shadow)."""
+    Pm32 = np.ascontiguousarray(Pm32, dtype=np.float32)
+    models = np.ascontiguousarray(models, dtype=np.int32)
+    gpu_of = np.ascontiguousarray(gpu_of, dtype=np.int32)
+    c64 = C.c_double(0)
+    _lib().oracle_assignment_cost.restype = C.c_float
+    c = _lib().oracle_assignment_cost(_p(Pm32), C.c_uint32(Pm32.shape[0]), _p(models), C.c_uint32(len(models)),
+                                      _p(gpu_of), C.byref(c64))
+    return np.float32(c), c64.value
+
+
+def optimal_assignment(Pm32, models, num_gpus, max_residents):
+    """Exhaustive search; returns (lowest cost float32, one optimal assignment, assignments tried)."""
+    Pm32 = np.ascontiguousarray(Pm32, dtype=np.float32)
+    models = np.ascontiguousarray(models, dtype=np.int32)
+    best = np.full(len(models), -1, dtype=np.int32)
+    tried = C.c_uint64(0)
+    _lib().oracle_optimal_assignment.restype = C.c_float
+    c = _lib().oracle_optimal_assignment(_p(Pm32), C.c_uint32(Pm32.shape[0]), _p(models), C.c_uint32(len(models)),
+                                         C.c_uint32(num_gpus), C.c_uint32(max_residents), _p(best), C.byref(tried))
+    return np.float32(c), best, int(tried.value)

@@ -462,3 +462,67 @@ void oracle_place(const float *Pm, uint32_t P, uint32_t G, uint32_t R,
     *tick += n;
     free(mu); free(mu64); free(admit64_g); free(score64_g);
 }
+
+/* ------------------------------------------------------------------ *
+ * Placement quality (Section 5, "Deployment accuracy evaluation against
+ * optimal strategies"): the deployment of n models on G identical GPUs
+ * (at most R per GPU) with the lowest average predicted drop, found by
+ * trying every assignment.  With the pairwise-sum estimate of Algorithm 1
+ * the drop of model i is the sum of Pm[m_i][m_j] over the other models j
+ * on its GPU, so the average drop of a deployment is
+ *     cost = ( sum over i < j on the same GPU of (Pm[m_i][m_j] + Pm[m_j][m_i]) ) / n.
+ * The value is DEFINED in float32: each pair term is one float add, terms are
+ * accumulated model by model (j ascending, and for each j its partners
+ * i < j ascending), one division at the end; cost64 is the same in double.
+ * ------------------------------------------------------------------ */
+float oracle_assignment_cost(const float *Pm, uint32_t P, const int32_t *models, uint32_t n,
+                             const int32_t *gpu_of, double *cost64)
+{
+    float tot = 0.0f; double tot64 = 0.0;
+    for (uint32_t j = 1; j < n; ++j)
+        for (uint32_t i = 0; i < j; ++i) {
+            if (gpu_of[i] < 0 || gpu_of[i] != gpu_of[j]) continue;
+            const float a = Pm[(size_t)models[i] * P + models[j]], b = Pm[(size_t)models[j] * P + models[i]];
+            tot = tot + (a + b);
+            tot64 += (double)a + (double)b;
+        }
+    if (cost64) *cost64 = tot64 / (double)n;
+    return tot / (float)n;
+}
+
+/* every assignment of models 1..n-1 (model 0 sits on GPU 0: the GPUs are identical) */
+static void optimal_rec(const float *Pm, uint32_t P, const int32_t *models, uint32_t n, uint32_t G, uint32_t R,
+                        uint32_t k, int32_t *gpu_of, uint32_t *load, float *best, int32_t *best_assign,
+                        uint64_t *tried)
+{
+    if (k == n) {
+        const float c = oracle_assignment_cost(Pm, P, models, n, gpu_of, NULL);
+        ++*tried;
+        if (*best < 0.0f || c < *best) { *best = c; memcpy(best_assign, gpu_of, sizeof(int32_t) * n); }
+        return;
+    }
+    for (uint32_t g = 0; g < G; ++g) {
+        if (load[g] >= R) continue;
+        gpu_of[k] = (int32_t)g; ++load[g];
+        optimal_rec(Pm, P, models, n, G, R, k + 1, gpu_of, load, best, best_assign, tried);
+        --load[g];
+    }
+}
+
+/* returns the lowest cost (float32) over all feasible assignments, -1 if none exists (n > G*R);
+ * best_assign[n] gets one optimal assignment (the first found in lexicographic order), tried the count */
+float oracle_optimal_assignment(const float *Pm, uint32_t P, const int32_t *models, uint32_t n,
+                                uint32_t G, uint32_t R, int32_t *best_assign, uint64_t *tried)
+{
+    int32_t *gpu_of = (int32_t *)malloc(sizeof(int32_t) * (n + 1));
+    uint32_t *load = (uint32_t *)calloc(G + 1, sizeof(uint32_t));
+    float best = -1.0f;
+    uint64_t t = 0;
+    if (n > 0 && R > 0 && G > 0) {
+        gpu_of[0] = 0; load[0] = 1;
+        optimal_rec(Pm, P, models, n, G, R, 1, gpu_of, load, &best, best_assign, &t);
+    }
+    if (tried) *tried = t;
+    free(gpu_of); free(load);
+    return best;
+}
