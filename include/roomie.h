@@ -273,6 +273,31 @@ int roomie_place_batch(const float *Pmat, uint32_t P, const roomie_cluster_state
                        const roomie_opts *opts /* host */, int32_t *gpu_out, float *mean_out, float *mu_arr_out,
                        void *stream);
 
+/* Placement quality (Section 5, "Deployment accuracy evaluation against optimal strategies"): for each of
+ * num_scenarios model lists, the deployment of its n models on num_gpus identical GPUs, at most
+ * max_residents per GPU, with the lowest average predicted drop - found by trying every assignment
+ * (model 0 fixed on GPU 0).  With the pairwise-sum estimate of Algorithm 1 the average drop is
+ *     cost = ( sum over i < j on the same GPU of (Pmat[m_i][m_j] + Pmat[m_j][m_i]) ) / n,
+ * evaluated in float32: one add per pair term, terms accumulated model by model (j ascending, its
+ * partners i < j ascending), one division.
+ *   models      [S][n] profile ids (duplicates = replicas)
+ *   best_cost   [S] lowest cost, -1 when n > num_gpus * max_residents
+ *   best_assign [S][n] optional: GPU of every model in the optimal deployment that comes first in
+ *               lexicographic order of (GPU of model 1, GPU of model 2, ...)
+ *   workspace   roomie_optimal_workspace_bytes(S) bytes of device scratch
+ * Limits: n <= 16, num_gpus <= 15, max_residents <= 15, num_gpus^(n-1) <= 2^32, S <= 65535
+ * (INVALID_ARG / CAPACITY otherwise). */
+size_t roomie_optimal_workspace_bytes(uint32_t num_scenarios);
+int roomie_optimal_assignment(const float *Pmat, uint32_t P, const int32_t *models, uint32_t n,
+                              uint32_t num_scenarios, uint32_t num_gpus, uint32_t max_residents,
+                              float *best_cost, int32_t *best_assign, void *workspace, size_t workspace_bytes,
+                              void *stream);
+
+/* The same cost for GIVEN deployments (e.g. the one Algorithm 2 arrived at): gpu_of [S][n], a negative
+ * entry = model not deployed (it takes part in no term but still counts in n). */
+int roomie_assignment_cost(const float *Pmat, uint32_t P, const int32_t *models, const int32_t *gpu_of,
+                           uint32_t n, uint32_t num_scenarios, float *cost_out, void *stream);
+
 /* Text of a roomie_status; the last CUDA error code/text seen by this thread's calls. */
 const char *roomie_strerror(int status);
 const char *roomie_last_cuda_error(void);

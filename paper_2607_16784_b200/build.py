@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libroomie.so")
-SOURCES = ["roomie_api.cu", "roomie_library.cu", "roomie_pairs.cu", "roomie_place.cu"]
+SOURCES = ["roomie_api.cu", "roomie_library.cu", "roomie_pairs.cu", "roomie_place.cu", "roomie_optimal.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=true", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

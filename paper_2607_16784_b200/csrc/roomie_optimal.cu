@@ -1,0 +1,177 @@
+// Placement quality (Section 5, "Deployment accuracy evaluation against optimal strategies"): the
+// deployment of n models on G identical GPUs with the lowest average predicted drop, by trying every
+// assignment - the optimum Algorithm 2's decisions are compared with.
+//
+// With the pairwise-sum estimate the average drop of a deployment is
+//     cost = ( sum over i < j on the same GPU of (P[m_i][m_j] + P[m_j][m_i]) ) / n,
+// defined in float32: pair terms are accumulated model by model (j ascending, partners i < j
+// ascending), one division at the end.  That order lets the search share work: a thread fixes the
+// GPUs of models 1..n-2 (model 0 sits on GPU 0), sums their terms once, and only adds the last
+// model's terms for each of its G choices.
+#include "roomie_common.cuh"
+
+namespace roomie {
+
+constexpr int kOptThreads = 256;
+constexpr int kOptMaxModels = 16;
+
+struct OptArgs {
+    const float* Pm;
+    uint32_t P;
+    const int32_t* models;          // [S][n]
+    uint32_t n, S, G, R;
+    unsigned long long* best_key;   // [S] (cost bits << 32) | code, smaller is better
+    unsigned long long n_prefix;    // G^(n-2) (1 when n <= 2)
+};
+
+// pair sums s[i][j] = P[m_i][m_j] + P[m_j][m_i] of one scenario into shared memory
+__device__ __forceinline__ void load_pair_sums(const OptArgs& g, const int32_t* models, float* s_pair) {
+    for (uint32_t t = threadIdx.x; t < g.n * g.n; t += blockDim.x) {
+        const uint32_t i = t / g.n, j = t % g.n;
+        const int32_t mi = models[i], mj = models[j];
+        s_pair[t] = __fadd_rn(__ldg(&g.Pm[(size_t)mi * g.P + mj]), __ldg(&g.Pm[(size_t)mj * g.P + mi]));
+    }
+}
+
+// grid: (CTAs per scenario, S)
+__global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs g) {
+    __shared__ float s_pair[kOptMaxModels * kOptMaxModels];
+    __shared__ unsigned long long s_best[kOptThreads / 32];
+    const uint32_t sc = blockIdx.y, n = g.n, G = g.G, R = g.R;
+    load_pair_sums(g, g.models + (size_t)sc * n, s_pair);
+    __syncthreads();
+    unsigned long long best = ~0ull;
+    const float fn = (float)n;
+    for (unsigned long long pc = (unsigned long long)blockIdx.x * kOptThreads + threadIdx.x; pc < g.n_prefix;
+         pc += (unsigned long long)gridDim.x * kOptThreads) {
+        // digits of the prefix code: model 1 is the most significant one; 4 bits per model / per GPU load
+        unsigned long long assign = 0, load = 1;                    // model 0 on GPU 0
+        unsigned long long rest = pc;
+        bool ok = true;
+        for (int k = (int)n - 2; k >= 1; --k) {
+            const uint32_t d = (uint32_t)(rest % G);
+            rest /= G;
+            assign |= (unsigned long long)d << (4 * k);
+            load += 1ull << (4 * d);
+        }
+        for (uint32_t d = 0; d < G; ++d) ok = ok && ((load >> (4 * d)) & 15ull) <= R;
+        if (!ok) continue;
+        float tot = 0.0f;                                           // terms among models 0 .. n-2
+        for (uint32_t j = 1; j + 1 < n; ++j) {
+            const uint32_t gj = (uint32_t)(assign >> (4 * j)) & 15u;
+            for (uint32_t i = 0; i < j; ++i)
+                if (((uint32_t)(assign >> (4 * i)) & 15u) == gj) tot = __fadd_rn(tot, s_pair[i * n + j]);
+        }
+        if (n == 1) {
+            best = 0ull;                                            // a single model: cost 0, code 0
+            continue;
+        }
+        for (uint32_t d = 0; d < G; ++d) {                          // the last model's GPU
+            if (((load >> (4 * d)) & 15ull) >= R) continue;
+            float c = tot;
+            for (uint32_t i = 0; i + 1 < n; ++i)
+                if (((uint32_t)(assign >> (4 * i)) & 15u) == d) c = __fadd_rn(c, s_pair[i * n + (n - 1)]);
+            const unsigned long long code = pc * G + d;
+            const unsigned long long key = ((unsigned long long)__float_as_uint(__fdiv_rn(c, fn)) << 32) | code;
+            best = key < best ? key : best;
+        }
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) {
+        const unsigned long long o = __shfl_xor_sync(0xffffffffu, best, s);
+        best = o < best ? o : best;
+    }
+    if ((threadIdx.x & 31) == 0) s_best[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kOptThreads / 32; ++w) best = s_best[w] < best ? s_best[w] : best;
+        if (best != ~0ull) atomicMin(&g.best_key[sc], best);
+    }
+}
+
+// best_key -> cost and assignment per scenario
+__global__ void optimal_unpack_kernel(const unsigned long long* best_key, uint32_t S, uint32_t n, uint32_t G,
+                                      float* best_cost, int32_t* best_assign) {
+    const uint32_t sc = blockIdx.x * blockDim.x + threadIdx.x;
+    if (sc >= S) return;
+    const unsigned long long key = best_key[sc];
+    if (key == ~0ull) {                                             // no feasible deployment
+        best_cost[sc] = -1.0f;
+        if (best_assign) for (uint32_t k = 0; k < n; ++k) best_assign[(size_t)sc * n + k] = -1;
+        return;
+    }
+    best_cost[sc] = __uint_as_float((uint32_t)(key >> 32));
+    if (best_assign) {
+        unsigned long long code = key & 0xffffffffull;
+        best_assign[(size_t)sc * n] = 0;
+        for (uint32_t k = n - 1; k >= 1; --k) { best_assign[(size_t)sc * n + k] = (int32_t)(code % G); code /= G; }
+    }
+}
+
+// cost of given deployments, one thread per scenario; gpu_of < 0 = model not deployed
+__global__ void assignment_cost_kernel(const float* __restrict__ Pm, uint32_t P, const int32_t* __restrict__ models,
+                                       const int32_t* __restrict__ gpu_of, uint32_t n, uint32_t S, float* cost) {
+    const uint32_t sc = blockIdx.x * blockDim.x + threadIdx.x;
+    if (sc >= S) return;
+    const int32_t* m = models + (size_t)sc * n;
+    const int32_t* a = gpu_of + (size_t)sc * n;
+    float tot = 0.0f;
+    for (uint32_t j = 1; j < n; ++j)
+        for (uint32_t i = 0; i < j; ++i)
+            if (a[i] >= 0 && a[i] == a[j])
+                tot = __fadd_rn(tot, __fadd_rn(__ldg(&Pm[(size_t)m[i] * P + m[j]]), __ldg(&Pm[(size_t)m[j] * P + m[i]])));
+    cost[sc] = __fdiv_rn(tot, (float)n);
+}
+
+}  // namespace roomie
+
+using namespace roomie;
+
+extern "C" size_t roomie_optimal_workspace_bytes(uint32_t num_scenarios) { return 8 * (size_t)num_scenarios + 256; }
+
+extern "C" int roomie_optimal_assignment(const float* Pmat, uint32_t P, const int32_t* models, uint32_t n,
+                                         uint32_t num_scenarios, uint32_t num_gpus, uint32_t max_residents,
+                                         float* best_cost, int32_t* best_assign, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+    if (!Pmat || P == 0 || !models || !best_cost || !workspace || n == 0 || n > kOptMaxModels || num_gpus == 0 ||
+        num_gpus > 15 || max_residents == 0 || max_residents > 15)
+        return ROOMIE_ERR_INVALID_ARG;
+    if (num_scenarios == 0) return ROOMIE_OK;
+    if (workspace_bytes < roomie_optimal_workspace_bytes(num_scenarios)) return ROOMIE_ERR_CAPACITY;
+    // the code of an assignment (base-G digits of models 1..n-1) must fit 32 bits
+    unsigned long long codes = 1, prefix = 1;
+    for (uint32_t k = 1; k < n; ++k) {
+        codes *= num_gpus;
+        if (k + 1 < n) prefix *= num_gpus;
+        if (codes > (1ull << 32)) return ROOMIE_ERR_CAPACITY;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned long long* keys = static_cast<unsigned long long*>(workspace);
+    ROOMIE_CUDA_OK(cudaMemsetAsync(keys, 0xFF, 8 * (size_t)num_scenarios, st));
+    OptArgs a;
+    a.Pm = Pmat; a.P = P; a.models = models; a.n = n; a.S = num_scenarios; a.G = num_gpus; a.R = max_residents;
+    a.best_key = keys; a.n_prefix = prefix;
+    unsigned long long ctas = (prefix + kOptThreads - 1) / kOptThreads;
+    const unsigned long long cap = (unsigned long long)sm_count() * 8;      // enough CTAs to fill the GPU per scenario
+    if (ctas > cap) ctas = cap;
+    if (num_scenarios > 65535) return ROOMIE_ERR_CAPACITY;
+    optimal_assignment_kernel<<<dim3((unsigned)ctas, num_scenarios), kOptThreads, 0, st>>>(a);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+    optimal_unpack_kernel<<<(num_scenarios + 127) / 128, 128, 0, st>>>(keys, num_scenarios, n, num_gpus, best_cost,
+                                                                       best_assign);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+    return ROOMIE_OK;
+}
+
+extern "C" int roomie_assignment_cost(const float* Pmat, uint32_t P, const int32_t* models, const int32_t* gpu_of,
+                                      uint32_t n, uint32_t num_scenarios, float* cost_out, void* stream) {
+    if (!Pmat || P == 0 || !models || !gpu_of || !cost_out || n == 0) return ROOMIE_ERR_INVALID_ARG;
+    if (num_scenarios == 0) return ROOMIE_OK;
+    assignment_cost_kernel<<<(num_scenarios + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        Pmat, P, models, gpu_of, n, num_scenarios, cost_out);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+    return ROOMIE_OK;
+}

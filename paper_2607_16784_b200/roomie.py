@@ -17,7 +17,8 @@ EXPORTS = [
     "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
     "roomie_pair_interference_static",
-    "roomie_multi_estimate", "roomie_place", "roomie_place_batch", "roomie_strerror", "roomie_last_cuda_error",
+    "roomie_multi_estimate", "roomie_place", "roomie_place_batch", "roomie_optimal_workspace_bytes",
+    "roomie_optimal_assignment", "roomie_assignment_cost", "roomie_strerror", "roomie_last_cuda_error",
     "roomie_launch_count", "roomie_reset_launch_count", "roomie_profile_enable", "roomie_profile_walk_ms",
 ]
 
@@ -48,6 +49,12 @@ def _load():
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     dll.roomie_pair_interference_static.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
                                                     C.c_void_p, C.c_void_p, C.c_void_p]
+    dll.roomie_optimal_workspace_bytes.restype = C.c_size_t
+    dll.roomie_optimal_workspace_bytes.argtypes = [C.c_uint32]
+    dll.roomie_optimal_assignment.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32,
+                                              C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    dll.roomie_assignment_cost.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32,
+                                           C.c_void_p, C.c_void_p]
     dll.roomie_occupancy.argtypes = [C.c_void_p] * 4
     dll.roomie_library_build.argtypes = [C.c_void_p] * 5
     dll.roomie_multi_estimate.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -383,6 +390,31 @@ def place_batch(Pmat, num_gpus, max_residents, ids, expiry, count, tick, arr_id,
     _check(_dll.roomie_place_batch(_ptr(Pm), Pm.shape[0], C.byref(state), _ptr(aid), _ptr(life), n, S, C.byref(o),
                                    _ptr(gpu), _ptr(mean), _ptr(mu_arr), _stream(stream)), "roomie_place_batch")
     return gpu, mean, mu_arr, dict(ids=ids_t, expiry=exp_t, count=cnt_t, tick=tick_t)
+
+
+def optimal_assignment(Pmat, models, num_gpus, max_residents, want_assign=True, stream=None):
+    """roomie_optimal_assignment: models [S, n] -> (best_cost float32 [S], best_assign int32 [S, n] or None)."""
+    Pm = _dev(Pmat, torch.float32)
+    m = _dev(models, torch.int32)
+    S, n = m.shape
+    cost = torch.empty(S, dtype=torch.float32, device=Pm.device)
+    assign = torch.empty((S, n), dtype=torch.int32, device=Pm.device) if want_assign else None
+    ws = _workspace(_dll.roomie_optimal_workspace_bytes(S), Pm.device)
+    _check(_dll.roomie_optimal_assignment(_ptr(Pm), Pm.shape[0], _ptr(m), n, S, int(num_gpus), int(max_residents),
+                                          _ptr(cost), _ptr(assign), _ptr(ws), ws.numel(), _stream(stream)),
+           "roomie_optimal_assignment")
+    return cost, assign
+
+
+def assignment_cost(Pmat, models, gpu_of, stream=None):
+    """roomie_assignment_cost: average predicted drop of given deployments, float32 [S]."""
+    Pm = _dev(Pmat, torch.float32)
+    m, a = _dev(models, torch.int32), _dev(gpu_of, torch.int32)
+    S, n = m.shape
+    cost = torch.empty(S, dtype=torch.float32, device=Pm.device)
+    _check(_dll.roomie_assignment_cost(_ptr(Pm), Pm.shape[0], _ptr(m), _ptr(a), n, S, _ptr(cost), _stream(stream)),
+           "roomie_assignment_cost")
+    return cost
 
 
 def launch_count() -> int:
