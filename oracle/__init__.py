@@ -22,6 +22,7 @@ _SRC = os.path.join(_HERE, "roomie_oracle.c")
 _LIB = os.path.join(_HERE, "libroomie_oracle.so")
 
 TIMELINE, LOCKSTEP = 0, 1
+DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS = 2, 3, 4
 
 
 def build(force: bool = False) -> str:

@@ -189,6 +189,121 @@ static void walk(const prof_view *A, const prof_view *B, uint32_t si, uint32_t s
     *delta_i = di; *delta_j = dj; *V = v; *evals = ev;
 }
 
+/* ------------------------------------------------------------------ *
+ * Section 3.2 in full ("Adjusted occupancy", "Two-phase execution",
+ * "Performance drop") for one alignment: the two kernel sequences are run
+ * together from (s_i, s_j); whenever the two active kernels' combined demand
+ * exceeds the SM (Eq. 2) each runs with the blocks b~ the partition policy
+ * leaves it, i.e. at occupancy o~ = W_b * b~ / W, and progresses at the rate
+ * o~/o = b~/b (its execution time is inversely proportional to its adjusted
+ * occupancy); the interference ends when the first of the two completes, and
+ * the other continues at full occupancy with what is left of it (two-phase
+ * execution), possibly against the finished model's next kernel.  Idle gaps
+ * between kernels are not stretched.  The delay of a model is the time its
+ * kernels took beyond their isolated durations; the run ends when either
+ * model has completed its last kernel.
+ *
+ * Policies for b~ (the paper names them, it does not spell them out):
+ *   2 EQUAL    each kernel may use half of every SM resource;
+ *   3 PRIORITY model i's kernel keeps its blocks, model j's kernel gets what
+ *              is left of every resource;
+ *   4 FCFS     the same with priority to the kernel that started earlier
+ *              (model i on a tie).
+ * A kernel left without a single block waits (rate 0) while the other runs
+ * at full occupancy; under EQUAL, when neither fits into half an SM, the
+ * kernel that started earlier (model i on a tie) runs alone.
+ * Per-block demands come from phi at the resident block count b.
+ * ------------------------------------------------------------------ */
+typedef struct { uint64_t wb, regs, smem, b; } block_need;
+
+static block_need need_of(const prof_view *p, uint32_t k)
+{
+    block_need n;
+    n.b = p->phi[3 * p->phi_stride + k];
+    n.wb = n.b ? p->phi[0 * p->phi_stride + k] / n.b : 0;
+    n.regs = n.b ? p->phi[1 * p->phi_stride + k] / n.b : 0;
+    n.smem = n.b ? p->phi[2 * p->phi_stride + k] / n.b : 0;
+    return n;
+}
+
+/* blocks of a kernel that fit into the given amounts of the four resources, at most its own b */
+static uint64_t blocks_in(const block_need *n, uint64_t warps, uint64_t regs, uint64_t smem, uint64_t slots)
+{
+    uint64_t b = n->b;
+    if (n->wb && warps / n->wb < b) b = warps / n->wb;
+    if (n->regs && regs / n->regs < b) b = regs / n->regs;
+    if (n->smem && smem / n->smem < b) b = smem / n->smem;
+    if (slots < b) b = slots;
+    return b;
+}
+
+static void walk_detailed(const prof_view *A, const prof_view *B, uint32_t si, uint32_t sj,
+                          const uint64_t cap[4], int policy,
+                          double *delta_i, double *delta_j, uint64_t *V, uint64_t *evals)
+{
+    uint32_t k[2] = { si, sj };
+    const prof_view *M[2] = { A, B };
+    double work[2], gap[2] = { 0.0, 0.0 }, began[2] = { 0.0, 0.0 }, lost[2] = { 0.0, 0.0 };
+    double now = 0.0, both = 0.0;
+    uint64_t ev = 0;
+    work[0] = A->dt[si]; work[1] = B->dt[sj];
+    while (k[0] < A->q && k[1] < B->q) {
+        ++ev;
+        double rate[2] = { 1.0, 1.0 };
+        const int active0 = gap[0] <= 0.0, active1 = gap[1] <= 0.0;
+        int contend = 0;
+        if (active0 && active1 && A->phi[k[0]] > 0 && B->phi[k[1]] > 0 && interferes(A, k[0], B, k[1], cap)) {
+            const block_need n0 = need_of(A, k[0]), n1 = need_of(B, k[1]);
+            uint64_t b0, b1;
+            contend = 1;
+            if (policy == 2) {
+                b0 = blocks_in(&n0, cap[0] / 2, cap[1] / 2, cap[2] / 2, cap[3] / 2);
+                b1 = blocks_in(&n1, cap[0] / 2, cap[1] / 2, cap[2] / 2, cap[3] / 2);
+                if (b0 == 0 && b1 == 0) { if (began[0] <= began[1]) b0 = n0.b; else b1 = n1.b; }
+                else if (b0 == 0) b1 = n1.b;
+                else if (b1 == 0) b0 = n0.b;
+            } else {
+                const int first = (policy == 3 || began[0] <= began[1]) ? 0 : 1;
+                const block_need *hi = first == 0 ? &n0 : &n1, *lo = first == 0 ? &n1 : &n0;
+                const uint64_t bl = blocks_in(lo, cap[0] - hi->wb * hi->b, cap[1] - hi->regs * hi->b,
+                                              cap[2] - hi->smem * hi->b, cap[3] - hi->b);
+                b0 = first == 0 ? n0.b : bl;
+                b1 = first == 0 ? bl : n1.b;
+            }
+            rate[0] = (double)b0 / (double)n0.b;
+            rate[1] = (double)b1 / (double)n1.b;
+        }
+        /* time to the next event: a kernel completes or a gap ends */
+        double t[2];
+        for (int m = 0; m < 2; ++m)
+            t[m] = gap[m] > 0.0 ? gap[m] : (rate[m] > 0.0 ? work[m] / rate[m] : INFINITY);
+        const double dt = t[0] < t[1] ? t[0] : t[1];
+        now += dt;
+        if (contend) both += dt;
+        for (int m = 0; m < 2; ++m) {
+            if (gap[m] > 0.0) {
+                gap[m] = t[m] <= dt ? 0.0 : gap[m] - dt;
+                if (gap[m] <= 0.0) began[m] = now;
+                continue;
+            }
+            lost[m] += dt * (1.0 - rate[m]);
+            if (t[m] <= dt) {                                   /* this kernel completes */
+                const prof_view *p = M[m];
+                const uint32_t done = k[m]++;
+                if (k[m] < p->q) {
+                    gap[m] = (double)p->start[k[m]] - ((double)p->start[done] + (double)p->dt[done]);
+                    work[m] = p->dt[k[m]];
+                    if (gap[m] <= 0.0) { gap[m] = 0.0; began[m] = now; }
+                }
+            } else {
+                work[m] -= dt * rate[m];
+            }
+        }
+    }
+    (void)both;
+    *delta_i = lost[0]; *delta_j = lost[1]; *V = 0; *evals = ev;   /* V is not defined in this mode */
+}
+
 static int cmp_double(const void *x, const void *y)
 {
     double a = *(const double *)x, b = *(const double *)y;
@@ -267,7 +382,8 @@ uint32_t oracle_pair(const oracle_library *L, uint32_t a, uint32_t b,
                 !(A.phi[si] > 0 && B.phi[sj] > 0 && interferes(&A, si, &B, sj, cap)))
                 continue;                        /* not an interference starting point */
             double di, dj; uint64_t v, ev;
-            walk(&A, &B, si, sj, cap, mode, &di, &dj, &v, &ev);
+            if (mode >= 2) walk_detailed(&A, &B, si, sj, cap, mode, &di, &dj, &v, &ev);
+            else walk(&A, &B, si, sj, cap, mode, &di, &dj, &v, &ev);
             if (kept < cap_align) {
                 if (out_si) out_si[kept] = si;
                 if (out_sj) out_sj[kept] = sj;
