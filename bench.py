@@ -54,7 +54,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="roomie", choices=["roomie", "reference"])
     ap.add_argument("--config", type=int, default=3, help="library configuration (0-4)")
-    ap.add_argument("--setting", default="base", choices=["base", "greedy", "lockstep_full"],
+    ap.add_argument("--setting", default="base", choices=["base", "greedy", "lockstep_full", "detailed"],
                     help="base: alignment (0,0); greedy: 8x8 alignments, start filter, median; lockstep_full: "
                          "Algorithm 1 as printed over the full Cartesian alignment set (use configs 1, 2 or 4)")
     ap.add_argument("--arrivals", type=int, default=10000)
@@ -67,12 +67,14 @@ def parse_args():
 def setting_kw(name):
     if name == "lockstep_full":
         return dict(mode=1, n_align=0, start_filter=1)
+    if name == "detailed":                              # Section 3.2 simulator, equal partition, alignment (0, 0)
+        return dict(mode=2, n_align=1, start_filter=0)
     return dict(mode=0, n_align=1, start_filter=0) if name == "base" else dict(mode=0, n_align=8, start_filter=1)
 
 
 def oracle_sample_pairs(setting, total_pairs):
     """Pairs the CPU oracle is timed on: all of them at the base setting, a bounded prefix otherwise."""
-    if setting == "base":
+    if setting in ("base", "detailed"):
         return total_pairs
     return max(1, total_pairs // (32 if setting == "greedy" else 512))
 
@@ -361,7 +363,7 @@ def main():
                     "ms_per_step": ms_e2e / args.steps},
             "gpu_launches": int(launches),
             "clocks": clocks,
-            "roofline": roofline or {"bound": "hbm", "kernel": "lockstep_full_kernel" if args.setting == "lockstep_full" else "timeline_tiles_kernel", "achieved": achieved, "peak": peak,
+            "roofline": roofline or {"bound": "hbm", "kernel": {"lockstep_full": "lockstep_full_kernel", "detailed": "detailed_walk_kernel"}.get(args.setting, "timeline_tiles_kernel"), "achieved": achieved, "peak": peak,
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": alg / launches_per_matrix if walk_launches else None,
                          "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix,

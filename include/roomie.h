@@ -129,6 +129,19 @@ int roomie_library_build(const roomie_library *lib /* host */, const roomie_kern
                                   only the time both kernels overlap is charged                  */
 #define ROOMIE_WALK_LOCKSTEP 1 /* Algorithm 1 as printed: both indices advance together, the whole
                                   duration d_k is charged                                        */
+/* Section 3.2 in full instead of Algorithm 1's closed-form delay: adjusted occupancy (a kernel that
+ * shares the SM runs with the blocks b~ the partition policy leaves it, at the rate o~/o = b~/b),
+ * two-phase execution (interference ends when the first of the two kernels completes), stretched
+ * timelines.  One value per partition policy the paper names:
+ *   EQUAL    each of the two kernels may use half of every SM resource;
+ *   PRIORITY the kernel of the pair's first model keeps its blocks, the other gets the remainder;
+ *   FCFS     the same with priority to the kernel that started earlier (first model on a tie).
+ * The alignment set, median, gamma and /T are applied as for the other modes; V is 0 and `evals`
+ * counts simulation events.  With PRIORITY, P[a][b] and P[b][a] of an unordered pair both come from
+ * the walk in which the lower-numbered profile has priority. */
+#define ROOMIE_WALK_DETAILED_EQUAL 2
+#define ROOMIE_WALK_DETAILED_PRIORITY 3
+#define ROOMIE_WALK_DETAILED_FCFS 4
 typedef struct roomie_opts {
     int32_t walk_mode;      /* ROOMIE_WALK_*                                                      */
     uint32_t n_align;       /* A: alignment set = A x A evenly spaced start indices floor(t*q/A);

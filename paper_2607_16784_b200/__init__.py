@@ -9,7 +9,7 @@ kernels.  PyTorch supplies device memory and streams, nothing else.
 There is no CPU fallback: importing this package without the compiled library raises.
 """
 from .roomie import (  # noqa: F401
-    GpuSpec, Library, ClusterState, RoomieError, TIMELINE, LOCKSTEP,
+    GpuSpec, Library, ClusterState, RoomieError, TIMELINE, LOCKSTEP, DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS,
     occupancy, library_build, pair_workspace_bytes, pair_matrix, pair_interference, pair_interference_static,
     multi_estimate, place, place_batch, optimal_assignment, assignment_cost, launch_count, reset_launch_count, profile_enable, profile_walk_ms, lib_path, EXPORTS,
 )

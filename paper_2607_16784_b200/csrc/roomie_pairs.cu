@@ -545,6 +545,7 @@ __global__ void __launch_bounds__(256) finalize_single_kernel(FinalArgs g) {
 }
 
 #include "roomie_lockstep_full.cuh"
+#include "roomie_detailed.cuh"
 
 // ---------------------------------------------------------------------------------------
 // host side
@@ -571,7 +572,8 @@ static bool batch_need(const roomie_library* lib, const roomie_opts* o, bool exp
     auto add = [&](uint32_t a, uint32_t b) {
         const uint32_t qa = off[a + 1] - off[a], qb = off[b + 1] - off[b];
         const uint64_t n = (uint64_t)host_grid_count(qa, o->n_align) * host_grid_count(qb, o->n_align);
-        const uint64_t per = o->walk_mode == ROOMIE_WALK_LOCKSTEP
+        const uint64_t per = o->walk_mode >= ROOMIE_WALK_DETAILED_EQUAL ? 1   // one result record per walk
+                             : o->walk_mode == ROOMIE_WALK_LOCKSTEP
                                  ? ((uint64_t)(qa < qb ? qa : qb) + kTileItems - 1) / kTileItems
                                  : ((uint64_t)qa + qb - 1 + kTileItems - 1) / kTileItems;
         tiles += n * per;
@@ -647,7 +649,7 @@ static int check_lib(const roomie_library* lib, const roomie_opts* o) {
     if (!lib || !o || !lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->share_table ||
         !lib->status || lib->num_profiles == 0)
         return ROOMIE_ERR_INVALID_ARG;
-    if (o->walk_mode != ROOMIE_WALK_TIMELINE && o->walk_mode != ROOMIE_WALK_LOCKSTEP) return ROOMIE_ERR_INVALID_ARG;
+    if (o->walk_mode < ROOMIE_WALK_TIMELINE || o->walk_mode > ROOMIE_WALK_DETAILED_FCFS) return ROOMIE_ERR_INVALID_ARG;
     return validate_spec(&lib->spec);
 }
 
@@ -667,6 +669,17 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
     lv.P = lib->num_profiles;
     lv.cap = make_cap(lib->spec);
 
+    if (o->walk_mode >= ROOMIE_WALK_DETAILED_EQUAL) {
+        // Section 3.2 simulator: one thread per walk writes its result where the tile partials go
+        DetailedArgs da;
+        da.lib = lv; da.ps = ps; da.slots = slots; da.n_align = o->n_align; da.start_filter = o->start_filter;
+        da.policy = o->walk_mode; da.spec = lib->spec; da.walks = walks; da.partials = partials;
+        profile_mark(st, true);
+        detailed_walk_kernel<<<(unsigned)((need.walks + 127) / 128), 128, 0, st>>>(da);
+        profile_mark(st, false);
+        note_launch();
+        ROOMIE_CUDA_OK(cudaGetLastError());
+    } else {
     PlanArgs pa;
     pa.lib = lv; pa.ps = ps; pa.slots = slots; pa.n_align = o->n_align; pa.start_filter = o->start_filter;
     pa.lockstep = o->walk_mode == ROOMIE_WALK_LOCKSTEP;
@@ -702,6 +715,7 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
     profile_mark(st, false);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
+    }
 
     FinalArgs fa;
     fa.lib = lv; fa.ps = ps; fa.slots = slots; fa.n_align = o->n_align; fa.walks = walks; fa.partials = partials;

@@ -12,6 +12,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_PKG, "libroomie.so")
 
 TIMELINE, LOCKSTEP = 0, 1
+DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS = 2, 3, 4
 
 EXPORTS = [
     "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",

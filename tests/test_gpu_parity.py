@@ -521,3 +521,49 @@ def test_placement_quality_experiment(rm, oracle):
     gap = float(((alg - opt) / np.maximum(opt, 1e-12)).mean())
     print(f"\n[placement quality] {S} scenarios, {n} models on {G} GPUs x {R}: Algorithm 2 matches the optimum in "
           f"{100 * match:.1f} % of them, mean relative gap {100 * gap:.2f} %")
+
+
+# ----------------------------------------------------------------------------- Section 3.2 simulator
+@pytest.mark.parametrize("mode", [2, 3, 4])
+def test_detailed_simulator_pair_detail(rm, oracle, mode):
+    """Adjusted occupancy + two-phase execution under the three partition policies, per alignment."""
+    from test_oracle_walk import tiny_lib
+    for feasible in (True, False):
+        lib = rs.make_library(0, feasible=feasible)
+        ol, gl = build_both(rm, oracle, lib)
+        for a, b in ((0, 1), (1, 0), (0, 0)):
+            for kw in (dict(n_align=1, start_filter=0), dict(n_align=8, start_filter=1), dict(n_align=0, start_filter=0)):
+                check_pair_detail(rm, oracle, ol, gl, a, b, mode=mode, **kw)
+    for seed in range(3):
+        lib = tiny_lib(seed, n_prof=3, qmax=9)
+        ol, gl = build_both(rm, oracle, lib)
+        for a in range(3):
+            for b in range(3):
+                check_pair_detail(rm, oracle, ol, gl, a, b, mode=mode, n_align=0, start_filter=0)
+
+
+@pytest.mark.parametrize("mode", [2, 3, 4])
+def test_detailed_simulator_matrices(rm, oracle, mode):
+    for cfg, kw in ((1, dict(n_align=1, start_filter=0)), (1, dict(n_align=8, start_filter=1)),
+                    (2, dict(n_align=8, start_filter=1)), (4, dict(n_align=1, start_filter=0))):
+        lib = rs.make_library(cfg)
+        ol, gl = build_both(rm, oracle, lib)
+        want, want_ev = oracle.pair_matrix(ol, mode=mode, **kw)
+        got, ev = rm.pair_matrix(gl, mode=mode, **kw)
+        assert int(ev.item()) == want_ev
+        assert_close(got.cpu().numpy(), want)
+
+
+def test_detailed_simulator_hand_cases_on_gpu(rm):
+    """The paper's two-phase formula straight through the CUDA path: a = 10 us, b = 30 us, both register-bound,
+    equal partition -> both at half rate until a ends at 20 us; b finishes alone at 40 us: each loses 10 us."""
+    from test_oracle_walk import make_lib
+    heavy = (256, 64, 0, 10000)
+    lib = make_lib([[heavy + (10.0, 0.0)], [heavy + (30.0, 0.0)]])
+    gl = rm.library_build(lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block,
+                          lib.dur_us, lib.gap_us, lib.offsets, lib.spec)
+    r = rm.pair_interference(gl, 0, 1, mode=2, detail_capacity=1)
+    assert float(r["delta_i"][0]) == 10000.0 and float(r["delta_j"][0]) == 10000.0
+    assert r["P2"].cpu().tolist() == [1.0, np.float32(1.0 / 3.0)]
+    r = rm.pair_interference(gl, 0, 1, mode=3, detail_capacity=1)          # priority: b waits for a
+    assert float(r["delta_i"][0]) == 0.0 and float(r["delta_j"][0]) == 10000.0
