@@ -39,33 +39,36 @@ struct OccResult {
     float occ, occ_theo;
 };
 
-// Section 3.1, Eq. 1 (see roomie_occupancy in roomie.h for the exact rules).
+// Section 3.1, Eq. 1 (see roomie_occupancy in roomie.h for the exact rules).  32-bit arithmetic: a
+// limit that would need more than 32 bits is a limit of zero blocks (the block does not fit).
 __device__ __forceinline__ OccResult occupancy_of(uint32_t grid, uint32_t threads, uint32_t regs,
                                                   uint32_t smem, const roomie_gpu_spec& s) {
     const uint32_t W = s.threads_per_sm / 32u;
-    const uint64_t Wb = ((uint64_t)threads + 31u) / 32u;
-    const uint64_t kInf = ~0ull;
-    const uint64_t regs_block = (uint64_t)regs * 32u * Wb;
-    uint64_t b = Wb ? (uint64_t)W / Wb : 0ull;
+    const uint32_t Wb = threads / 32u + ((threads & 31u) ? 1u : 0u);
+    const uint32_t kInf = 0xffffffffu;
+    uint32_t b = Wb ? W / Wb : 0u;                                   // warp limit
     uint32_t which = 0;
-    const uint64_t l1 = s.blocks_per_sm;
-    const uint64_t l2 = regs_block ? (uint64_t)s.regs_per_sm / regs_block : kInf;
-    const uint64_t l3 = smem ? (uint64_t)(s.smem_per_sm / smem) : kInf;
+    const uint32_t l1 = s.blocks_per_sm;                             // block-slot limit
+    // registers of one block = regs * 32 * Wb (threads padded to whole warps)
+    const unsigned long long regs_block64 = (unsigned long long)regs * 32u * Wb;
+    const uint32_t regs_block = regs_block64 > s.regs_per_sm ? 0u : (uint32_t)regs_block64;
+    const uint32_t l2 = regs_block64 == 0 ? kInf : (regs_block ? s.regs_per_sm / regs_block : 0u);
+    const uint32_t l3 = smem ? s.smem_per_sm / smem : kInf;
     if (l1 < b) { b = l1; which = 1; }
     if (l2 < b) { b = l2; which = 2; }
     if (l3 < b) { b = l3; which = 3; }
-    const uint64_t b_grid = ((uint64_t)grid + s.num_sms - 1u) / s.num_sms;
-    uint64_t br = b;
+    const uint32_t b_grid = grid ? (grid - 1u) / s.num_sms + 1u : 0u;
+    uint32_t br = b;
     if (b_grid < b) { br = b_grid; which = 4; }
     OccResult r;
-    r.b_lim = (uint32_t)b;
-    r.b_res = (uint32_t)br;
+    r.b_lim = b;
+    r.b_res = br;
     r.limiter = which;
-    r.warps = (uint32_t)(Wb * br);
-    r.phi_regs = (uint32_t)(br * regs_block);
-    r.phi_smem = (uint32_t)(br * smem);
+    r.warps = Wb * br;                                               // br <= W / Wb
+    r.phi_regs = br * regs_block;                                    // br <= R / regs_block (0 when br = 0)
+    r.phi_smem = br * smem;                                          // br <= S / smem
     r.occ = W ? __fdiv_rn((float)r.warps, (float)W) : 0.0f;
-    r.occ_theo = W ? __fdiv_rn((float)(uint32_t)(Wb * b), (float)W) : 0.0f;
+    r.occ_theo = W ? __fdiv_rn((float)(Wb * b), (float)W) : 0.0f;
     return r;
 }
 

@@ -29,12 +29,14 @@ __device__ __forceinline__ void occ_store_scalar(const OccArgs& a, uint32_t k, c
     }
 }
 
-template <bool kVec>
+// kVec: inputs and the packed / occ / occ_theo outputs are 16-byte aligned, so the first n/4*4 kernels go
+// four per thread with 128-bit accesses (the up to three left over are done one by one);
+// kVecPhi: n is a multiple of 4 as well, so the four component arrays of phi are aligned too.
+template <bool kVec, bool kVecPhi>
 __global__ void __launch_bounds__(256) occupancy_kernel(OccArgs a) {
     uint32_t bad = 0;
+    const uint32_t n4 = kVec ? a.n / 4 : 0;
     if (kVec) {
-        // n is a multiple of 4 and every array is 16-byte aligned in this variant
-        const uint32_t n4 = a.n / 4;
         for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x) {
             const uint4 g = __ldg(reinterpret_cast<const uint4*>(a.grid) + i);
             const uint4 t = __ldg(reinterpret_cast<const uint4*>(a.threads) + i);
@@ -61,19 +63,30 @@ __global__ void __launch_bounds__(256) occupancy_kernel(OccArgs a) {
                 reinterpret_cast<float4*>(a.occ_theo)[i] =
                     make_float4(o[0].occ_theo, o[1].occ_theo, o[2].occ_theo, o[3].occ_theo);
             if (a.phi) {
-                uint4* p = reinterpret_cast<uint4*>(a.phi);
-                p[i] = make_uint4(o[0].warps, o[1].warps, o[2].warps, o[3].warps);
-                p[n4 + i] = make_uint4(o[0].phi_regs, o[1].phi_regs, o[2].phi_regs, o[3].phi_regs);
-                p[2 * (size_t)n4 + i] = make_uint4(o[0].phi_smem, o[1].phi_smem, o[2].phi_smem, o[3].phi_smem);
-                p[3 * (size_t)n4 + i] = make_uint4(o[0].b_res, o[1].b_res, o[2].b_res, o[3].b_res);
+                if (kVecPhi) {
+                    uint4* p = reinterpret_cast<uint4*>(a.phi);
+                    p[i] = make_uint4(o[0].warps, o[1].warps, o[2].warps, o[3].warps);
+                    p[n4 + i] = make_uint4(o[0].phi_regs, o[1].phi_regs, o[2].phi_regs, o[3].phi_regs);
+                    p[2 * (size_t)n4 + i] = make_uint4(o[0].phi_smem, o[1].phi_smem, o[2].phi_smem, o[3].phi_smem);
+                    p[3 * (size_t)n4 + i] = make_uint4(o[0].b_res, o[1].b_res, o[2].b_res, o[3].b_res);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const size_t k = 4 * (size_t)i + j;
+                        a.phi[k] = o[j].warps;
+                        a.phi[(size_t)a.n + k] = o[j].phi_regs;
+                        a.phi[2 * (size_t)a.n + k] = o[j].phi_smem;
+                        a.phi[3 * (size_t)a.n + k] = o[j].b_res;
+                    }
+                }
             }
         }
-    } else {
-        for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < a.n; k += gridDim.x * blockDim.x) {
-            const OccResult o = occupancy_of(a.grid[k], a.threads[k], a.regs[k], a.smem[k], a.spec);
-            bad += (o.b_lim == 0);
-            occ_store_scalar(a, k, o);
-        }
+    }
+    // everything (scalar variant) or the tail after the last full group of four
+    for (uint32_t k = 4 * n4 + blockIdx.x * blockDim.x + threadIdx.x; k < a.n; k += gridDim.x * blockDim.x) {
+        const OccResult o = occupancy_of(a.grid[k], a.threads[k], a.regs[k], a.smem[k], a.spec);
+        bad += (o.b_lim == 0);
+        occ_store_scalar(a, k, o);
     }
     if (a.n_unlaunchable) {
 #pragma unroll
@@ -97,6 +110,7 @@ struct BuildArgs {
 };
 
 constexpr int kBuildThreads = 256;
+constexpr int kBuildItems = 4;                       // consecutive kernels per thread and trip
 
 __device__ __forceinline__ uint32_t to_ticks(float us, bool at_least_one, uint32_t& flags) {
     float f = __fmul_rn(us, 1000.0f);
@@ -113,16 +127,22 @@ __global__ void __launch_bounds__(kBuildThreads) library_build_kernel(BuildArgs 
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     unsigned long long carry = 0, sum_d = 0;
     uint32_t flags = 0;
-    for (uint32_t base = lo; base < hi; base += kBuildThreads) {
-        const uint32_t k = base + threadIdx.x;
-        const bool live = k < hi;
-        uint32_t dt = 0, gt = 0;
-        if (live) {
-            dt = to_ticks(a.dur_us[k], true, flags);
-            gt = to_ticks(a.gap_us[k], false, flags);
+    for (uint32_t base = lo; base < hi; base += kBuildThreads * kBuildItems) {
+        const uint32_t k0 = base + threadIdx.x * kBuildItems;
+        uint32_t dt[kBuildItems], gt[kBuildItems];
+        unsigned long long mine = 0, d = 0;
+#pragma unroll
+        for (int j = 0; j < kBuildItems; ++j) {
+            dt[j] = gt[j] = 0;
+            if (k0 + j < hi) {
+                dt[j] = to_ticks(a.dur_us[k0 + j], true, flags);
+                gt[j] = to_ticks(a.gap_us[k0 + j], false, flags);
+            }
+            mine += (unsigned long long)dt[j] + gt[j];
+            d += dt[j];
         }
-        // inclusive scan of (dt + gt) across the CTA
-        unsigned long long v = (unsigned long long)dt + gt, d = dt;
+        // inclusive scan of the per-thread sums across the CTA
+        unsigned long long v = mine;
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) {
             const unsigned long long up = __shfl_up_sync(0xffffffffu, v, s);
@@ -133,22 +153,26 @@ __global__ void __launch_bounds__(kBuildThreads) library_build_kernel(BuildArgs 
         if (lane == 31) warp_tot[wid] = v;
         if (lane == 0) warp_dur[wid] = d;
         __syncthreads();
-        unsigned long long before = carry, chunk = 0, chunk_d = 0;
+        unsigned long long start = carry + v - mine, chunk = 0, chunk_d = 0;
 #pragma unroll
         for (int w = 0; w < kBuildThreads / 32; ++w) {
-            if (w < wid) before += warp_tot[w];
+            if (w < wid) start += warp_tot[w];
             chunk += warp_tot[w];
             chunk_d += warp_dur[w];
         }
-        if (live) {
-            const unsigned long long start = before + v - ((unsigned long long)dt + gt);
-            const OccResult o = occupancy_of(a.grid[k], a.threads[k], a.regs[k], a.smem[k], a.spec);
-            uint4 rec;
-            rec.x = (uint32_t)start;
-            rec.y = (uint32_t)(start + dt);
-            rec.z = o.phi_regs | (o.warps << kWarpShift);
-            rec.w = o.phi_smem | (o.b_res << 22);
-            a.records[k] = rec;
+#pragma unroll
+        for (int j = 0; j < kBuildItems; ++j) {
+            const uint32_t k = k0 + j;
+            if (k < hi) {
+                const OccResult o = occupancy_of(a.grid[k], a.threads[k], a.regs[k], a.smem[k], a.spec);
+                uint4 rec;
+                rec.x = (uint32_t)start;
+                rec.y = (uint32_t)(start + dt[j]);
+                rec.z = o.phi_regs | (o.warps << kWarpShift);
+                rec.w = o.phi_smem | (o.b_res << 22);
+                a.records[k] = rec;
+                start += (unsigned long long)dt[j] + gt[j];
+            }
         }
         carry += chunk;
         sum_d += chunk_d;
@@ -195,15 +219,18 @@ extern "C" int roomie_occupancy(const roomie_kernel_table* table, const roomie_g
     a.packed4 = out->packed4; a.occ = out->occ; a.occ_theo = out->occ_theo; a.phi = out->phi;
     a.n_unlaunchable = out->n_unlaunchable;
     a.n = table->n; a.spec = *spec;
-    const bool vec = (a.n % 4 == 0) && aligned16(a.grid) && aligned16(a.threads) && aligned16(a.regs) &&
-                     aligned16(a.smem) && aligned16(a.packed4) && aligned16(a.occ) &&
-                     aligned16(a.occ_theo) && aligned16(a.phi);
+    // the 128-bit variant pays off only when phi can be stored with 128-bit accesses too (n a multiple of 4 or no
+    // phi output): four scalar stores per component at a 16-byte stride waste more than the wide loads gain
+    const bool vec_phi = (a.n % 4 == 0 || !a.phi) && aligned16(a.phi);
+    const bool vec = a.n >= 4 && vec_phi && aligned16(a.grid) && aligned16(a.threads) && aligned16(a.regs) &&
+                     aligned16(a.smem) && aligned16(a.packed4) && aligned16(a.occ) && aligned16(a.occ_theo);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint32_t work = vec ? a.n / 4 : a.n;
     uint32_t blocks = (work + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    if (vec) occupancy_kernel<true><<<blocks, 256, 0, st>>>(a);
-    else occupancy_kernel<false><<<blocks, 256, 0, st>>>(a);
+    if (vec_phi) occupancy_kernel<true, true><<<blocks, 256, 0, st>>>(a);
+    else if (vec) occupancy_kernel<true, false><<<blocks, 256, 0, st>>>(a);
+    else occupancy_kernel<false, false><<<blocks, 256, 0, st>>>(a);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;
