@@ -211,21 +211,23 @@ struct TileArgs {
 
 // Shared-memory layout of one tile.  The tile's A records sit at unified indices 0, 1, 2, ... and
 // its B records at kTop, kTop-1, ... (the two runs never meet: together they hold at most
-// kTileLoad <= kTop + 1 records).  Records are padded by one slot after every 8 so that the lanes of a
-// warp, whose positions on the merge path are about 8 records apart, fall into different bank
-// groups; the search keys (end ticks) live in their own array with one pad word per 32 so that
-// the binary-search probes of a warp do not collide either.  Both paddings are linear in the
-// staging loop's trip count, so staging addresses are base + immediate.
+// kTileLoad <= kTop + 1 records).  Records are padded by one slot after every 16 so that the lanes of a
+// warp, whose positions on the merge path are 16 steps apart, fall into different bank groups when
+// they read their 16-byte records (without padding the walk is 11 % slower; one slot per 8 costs a
+// resident CTA).  The padding is linear in the staging loop's trip count, so staging addresses are
+// base + immediate.  Nothing else lives in shared memory: the diagonal search probes the end ticks
+// inside the records, and the reciprocal of o_i + o_j comes from the special-function unit, which
+// leaves room for 6 resident CTAs (24 warps) per SM.
 // Staged A records carry the *slack* Phi|guards - phi_a in place of phi_a; B records keep phi_b:
 // Eq. 2 for a pairing is then two subtractions and a test of the guard bits.
-__device__ __forceinline__ uint32_t rec_slot(uint32_t i) { return i + (i >> 3); }
-__device__ __forceinline__ uint32_t key_slot(uint32_t i) { return i + (i >> 5); }
+constexpr int kPadShift = 4;
+__device__ __forceinline__ uint32_t rec_slot(uint32_t i) { return i + (i >> kPadShift); }
 constexpr int kTileLoad = kTileItems + 2;                               // one look-ahead record per side
 constexpr int kTop = ((kTileLoad + 31) / 32) * 32 + 31;                  // unified index of B[0]; = 31 mod 32 so that
                                                                          // a warp's descending run starts on a pad boundary
-constexpr int kRecSlots = kTop + (kTop >> 3) + 2;
-constexpr int kKeySlots = kTop + (kTop >> 5) + 2;
-constexpr int kStageBatch = 6;                                           // global loads in flight per thread
+constexpr int kRecSlots = kTop + (kTop >> kPadShift) + 2;
+constexpr int kTileCtasPerSm = 6;
+constexpr int kStageBatch = 3;                                           // global loads in flight per thread
 constexpr int kStageRounds = (kTileLoad + kTileThreads * kStageBatch - 1) / (kTileThreads * kStageBatch);
 
 template <bool kWithV>
@@ -259,14 +261,12 @@ __device__ __forceinline__ float small_int_to_float(uint32_t v) {
 // (step = +1 for A, -1 for B); kSlack: store cap - phi instead of phi
 template <bool kSlack, int kDir>
 __device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32_t n, uint32_t base_tick, PhiCap cap,
-                                           uint4* s_rec, int32_t* s_key) {
-    // thread t handles records t, t + 128, ...; 128 is a multiple of 8 and 32, so both paddings
-    // advance by a constant per trip
+                                           uint4* s_rec) {
+    // thread t handles records t, t + 128, ...; 128 is a multiple of the padding period, so the
+    // padded slot advances by a constant per trip
     const uint32_t i0 = kDir > 0 ? threadIdx.x : (uint32_t)kTop - threadIdx.x;
     uint4* rp = s_rec + rec_slot(i0);
-    int32_t* kp = s_key + key_slot(i0);
-    constexpr int kRecStep = kDir * (kTileThreads + kTileThreads / 8);
-    constexpr int kKeyStep = kDir * (kTileThreads + kTileThreads / 32);
+    constexpr int kRecStep = kDir * (kTileThreads + (kTileThreads >> kPadShift));
 #pragma unroll
     for (int round = 0; round < kStageRounds; ++round) {
         const uint32_t r0 = threadIdx.x + round * kStageBatch * kTileThreads;
@@ -281,20 +281,30 @@ __device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32
                 r[j].x -= base_tick; r[j].y -= base_tick;
                 if (kSlack) { r[j].z = cap.lo - r[j].z; r[j].w = cap.hi - r[j].w; }
                 rp[(round * kStageBatch + j) * kRecStep] = r[j];
-                kp[(round * kStageBatch + j) * kKeyStep] = (int32_t)r[j].y;
             }
         }
     }
 }
 
+// 1/x to one unit in the last place (special-function unit); the delay sums are float32 within
+// 1e-5 relative either way
+__device__ __forceinline__ float fast_rcp(float x) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
 // one step of the walk for the pairing (ra, rb).  A step that is not live (ragged tail of a walk)
 // touches nothing: the registers may then hold a record from beyond the staged range.
+// fa, fb: the two kernels' resident warps as floats (o = warps / W; W cancels in o_i / (o_i + o_j)).
+// Two kernels without a resident block never interfere, so the guard of the reciprocal only keeps
+// 0 * inf out of the sums.
 #define ROOMIE_WALK_STEP(live)                                                                         \
     if (live) {                                                                                        \
         const int32_t Ea = (int32_t)ra.y, Eb = (int32_t)rb.y;                                          \
         const int32_t ov = min(Ea, Eb) - max((int32_t)ra.x, (int32_t)rb.x);                            \
         const bool hit = (ov > 0) && phi_exceeds(ra.z, ra.w, rb.z, rb.w);                              \
-        const float tw = (hit ? (float)ov : 0.0f) * s_inv[wsum_b - wslack_a];   /* overlap/(o_i+o_j) */ \
+        const float tw = (hit ? (float)ov : 0.0f) * fast_rcp(fmaxf(fa + fb, 1.0f));  /* overlap/(o_i+o_j) */ \
         di = fmaf(tw, fa, di);                                                                         \
         dj = fmaf(tw, fb, dj);                                                                         \
         if (kWithV) V += hit ? (unsigned long long)(uint32_t)ov : 0ull;                                \
@@ -306,23 +316,20 @@ __device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32
         ib -= adv_a ? 0u : 1u;                                                                         \
         const uint4 r = s_rec[rec_slot(adv_a ? x : ib)];                                               \
         if (adv_a) {                                                                                   \
-            ra = r; wslack_a = r.z >> kWarpShift; fa = small_int_to_float(wconst - wslack_a);          \
+            ra = r; fa = small_int_to_float(wconst - (r.z >> kWarpShift));                             \
         } else {                                                                                       \
-            rb = r; wsum_b = (r.z >> kWarpShift) + wconst; fb = small_int_to_float(r.z >> kWarpShift); \
+            rb = r; fb = small_int_to_float(r.z >> kWarpShift);                                        \
         }                                                                                              \
     }
 
 template <bool kWithV>
-__global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArgs g) {
+__global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_kernel(TileArgs g) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint4* s_rec = reinterpret_cast<uint4*>(smem_raw);
-    int32_t* s_key = reinterpret_cast<int32_t*>(smem_raw + (size_t)kRecSlots * sizeof(uint4));
-    float* s_inv = reinterpret_cast<float*>(s_key + kKeySlots);
     __shared__ float s_f[2 * kTileThreads / 32];
     __shared__ unsigned long long s_v[kTileThreads / 32];
     __shared__ uint32_t s_t[kTileThreads / 32];
 
-    for (uint32_t i = threadIdx.x; i < g.n_inv; i += kTileThreads) s_inv[i] = __ldg(&g.inv_table[i]);
     const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
     // warps field of a staged A record holds (W + guard) - warps_a
     const uint32_t wconst = g.cap.lo >> kWarpShift;
@@ -331,8 +338,8 @@ __global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArg
         const TileDesc d = g.tiles[t];
         const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
         __syncthreads();                                   // previous tile fully consumed
-        stage_side<true, +1>(g.records + d.recA, loadA, d.baseA, g.cap, s_rec, s_key);
-        stage_side<false, -1>(g.records + d.recB, loadB, d.baseB, g.cap, s_rec, s_key);
+        stage_side<true, +1>(g.records + d.recA, loadA, d.baseA, g.cap, s_rec);
+        stage_side<false, -1>(g.records + d.recB, loadB, d.baseB, g.cap, s_rec);
         __syncthreads();
         const uint32_t len = d.cntA + d.cntB;
         const uint32_t diag = threadIdx.x * kItems;
@@ -346,12 +353,12 @@ __global__ void __launch_bounds__(kTileThreads, 4) timeline_tiles_kernel(TileArg
             const uint32_t btop = (uint32_t)(kTop + 1) - diag;             // index of B[diag - 1 - mid] is btop + mid
             while (lo < hi) {
                 const uint32_t mid = (lo + hi) >> 1;
-                if (s_key[key_slot(mid)] <= s_key[key_slot(btop + mid)]) lo = mid + 1; else hi = mid;
+                if ((int32_t)s_rec[rec_slot(mid)].y <= (int32_t)s_rec[rec_slot(btop + mid)].y) lo = mid + 1;
+                else hi = mid;
             }
             uint32_t x = lo, ib = (uint32_t)kTop - (diag - lo);
             uint4 ra = s_rec[rec_slot(x)], rb = s_rec[rec_slot(ib)];
-            uint32_t wslack_a = ra.z >> kWarpShift, wsum_b = (rb.z >> kWarpShift) + wconst;
-            float fa = small_int_to_float(wconst - wslack_a), fb = small_int_to_float(rb.z >> kWarpShift);
+            float fa = small_int_to_float(wconst - (ra.z >> kWarpShift)), fb = small_int_to_float(rb.z >> kWarpShift);
             if (len - diag >= (uint32_t)kItems) {
 #pragma unroll
                 for (int s = 0; s < kItems; ++s) ROOMIE_WALK_STEP(true)
@@ -700,14 +707,13 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
         if (grid > need.tiles) grid = need.tiles ? need.tiles : 1;
         lockstep_tiles_kernel<<<(unsigned)grid, kTileThreads, 0, st>>>(ta);
     } else {
-        const size_t smem = (size_t)kRecSlots * sizeof(uint4) + (size_t)kKeySlots * sizeof(int32_t) +
-                            (size_t)ta.n_inv * sizeof(float);
+        const size_t smem = (size_t)kRecSlots * sizeof(uint4);
         auto kern = detail ? timeline_tiles_kernel<true> : timeline_tiles_kernel<false>;
         if (smem > 48 * 1024)
             ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         // persistent grid: as many CTAs as fit at once, each striding over the tile list
-        int per_sm = (int)((227 * 1024) / (smem + 1024 + 256));
-        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
+        int per_sm = (int)((228 * 1024) / (smem + 1024 + 128));
+        per_sm = per_sm < 1 ? 1 : (per_sm > kTileCtasPerSm ? kTileCtasPerSm : per_sm);
         uint64_t grid = (uint64_t)sm_count() * per_sm;
         if (grid > need.tiles) grid = need.tiles ? need.tiles : 1;
         kern<<<(unsigned)grid, kTileThreads, smem, st>>>(ta);

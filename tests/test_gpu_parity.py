@@ -567,3 +567,30 @@ def test_detailed_simulator_hand_cases_on_gpu(rm):
     assert r["P2"].cpu().tolist() == [1.0, np.float32(1.0 / 3.0)]
     r = rm.pair_interference(gl, 0, 1, mode=3, detail_capacity=1)          # priority: b waits for a
     assert float(r["delta_i"][0]) == 0.0 and float(r["delta_j"][0]) == 10000.0
+
+
+# ----------------------------------------------------------------------------- size extremes
+def test_very_long_profiles_and_single_profile_library(rm, oracle):
+    """Profiles far longer than one tile (20 000 and 13 001 kernels: 17 tiles, ragged tail) and a library of one
+    profile (only the diagonal pair exists)."""
+    from types import SimpleNamespace
+    big = rs.make_library(3, num_profiles=16)
+    assert len(big.dur_us) >= 33001                                               # cut anew into two long profiles
+    src = {k: getattr(big, k)[:33001] for k in ("grid_blocks", "block_threads", "regs_per_thread", "smem_per_block")}
+    lib = SimpleNamespace(spec=big.spec, offsets=np.array([0, 20000, 33001], np.uint32),
+                          dur_us=(big.dur_us[:33001] * 0.2).astype(np.float32), gap_us=big.gap_us[:33001], **src)
+    ol, gl = build_both(rm, oracle, lib)
+    assert gl.status_flags() == 0
+    for kw in (dict(mode=0, n_align=1, start_filter=0), dict(mode=0, n_align=8, start_filter=1),
+               dict(mode=1, n_align=8, start_filter=0), dict(mode=2, n_align=1, start_filter=0)):
+        want, wev = oracle.pair_matrix(ol, **kw)
+        got, ev = rm.pair_matrix(gl, **kw)
+        assert int(ev.item()) == wev
+        assert_close(got.cpu().numpy(), want)
+    one = SimpleNamespace(spec=big.spec, offsets=np.array([0, 777], np.uint32), dur_us=big.dur_us[:777],
+                          gap_us=big.gap_us[:777], **{k: v[:777] for k, v in src.items()})
+    ol1, gl1 = build_both(rm, oracle, one)
+    want, wev = oracle.pair_matrix(ol1, mode=0, n_align=8, start_filter=1)
+    got, ev = rm.pair_matrix(gl1, mode=0, n_align=8, start_filter=1)
+    assert got.shape == (1, 1) and int(ev.item()) == wev
+    assert_close(got.cpu().numpy(), want)
