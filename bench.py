@@ -41,9 +41,9 @@ def walk_kernel_dram_bytes(num_kernels, evals, walks):
     """DRAM bytes (read + write) of one launch of the pairwise walk kernel.  Not measured on the full
     workload: the ncu capture of a small case (profiles/timeline_tiles_kernel_config3.md) shows
     compulsory first-touch reads only - 16 B per library record plus the 32 B descriptor of every tile
-    of 2048 path steps, partial results staying in L2 - and this model reproduces that capture
+    of 1536 path steps, partial results staying in L2 - and this model reproduces that capture
     (6.52 MB against 6.57 MB measured).  Every further read of a record is served by L2."""
-    tiles = evals / 2048.0 + walks / 2.0
+    tiles = evals / 1536.0 + walks / 2.0
     return int(16 * num_kernels + 32 * tiles)
 
 

@@ -206,8 +206,15 @@ typedef struct roomie_pair_detail {
     uint32_t *evals;   /* pairings scored by the walk                                */
 } roomie_pair_detail;
 
+/* Bytes of workspace roomie_pair_interference needs for the pair (a, b) under `opts` (with or
+ * without detail).  0 on invalid arguments or when the pair has more than 4096 alignments. */
+size_t roomie_pair_interference_workspace_bytes(const roomie_library *lib /* host */, uint32_t a, uint32_t b,
+                                                const roomie_opts *opts /* host */);
+
 /* The same computation for ONE ordered pair (a, b), any order, a == b allowed:
- * out2[0] = P[a][b], out2[1] = P[b][a].  `detail` (host struct) may be NULL. */
+ * out2[0] = P[a][b], out2[1] = P[b][a].  `detail` (host struct) may be NULL.  `workspace`: device,
+ * 256-byte aligned, at least roomie_pair_interference_workspace_bytes(lib, a, b, opts) bytes
+ * (ROOMIE_ERR_CAPACITY otherwise). */
 int roomie_pair_interference(const roomie_library *lib /* host */, uint32_t a, uint32_t b,
                              const roomie_opts *opts /* host */, float *out2, uint64_t *evals_out,
                              const roomie_pair_detail *detail, void *workspace, size_t workspace_bytes,

@@ -17,7 +17,7 @@
 namespace roomie {
 
 constexpr int kTileThreads = 128;
-constexpr int kItems = 16;                              // path steps per thread
+constexpr int kItems = 12;                              // path steps per thread
 constexpr int kTileItems = kTileThreads * kItems;       // path steps per tile
 
 struct PairSet {                  // which pairs a launch covers
@@ -207,28 +207,37 @@ struct TileArgs {
     const float* inv_table;      // [2W + 1] 1/s
     uint32_t n_inv;              // 2W + 1
     PhiCap cap;
+    uint32_t* status;            // library status word (sticky flags)
 };
 
 // Shared-memory layout of one tile.  The tile's A records sit at unified indices 0, 1, 2, ... and
-// its B records at kTop, kTop-1, ... (the two runs never meet: together they hold at most
-// kTileLoad <= kTop + 1 records).  Records are padded by one slot after every 16 so that the lanes of a
-// warp, whose positions on the merge path are 16 steps apart, fall into different bank groups when
-// they read their 16-byte records (without padding the walk is 11 % slower; one slot per 8 costs a
-// resident CTA).  The padding is linear in the staging loop's trip count, so staging addresses are
-// base + immediate.  Nothing else lives in shared memory: the diagonal search probes the end ticks
-// inside the records, and the reciprocal of o_i + o_j comes from the special-function unit, which
-// leaves room for 6 resident CTAs (24 warps) per SM.
-// Staged A records carry the *slack* Phi|guards - phi_a in place of phi_a; B records keep phi_b:
-// Eq. 2 for a pairing is then two subtractions and a test of the guard bits.
-constexpr int kPadShift = 4;
+// its B records at b_off, b_off + 1, ... with b_off the A count rounded up to a multiple of kChunk.
+// Nothing else lives in shared memory: the diagonal search probes the end ticks inside the records
+// and the reciprocal of o_i + o_j comes from the special-function unit, which leaves room for 8
+// resident CTAs (32 warps) per SM.
+//
+// Staging is done by the copy engine, not by the threads: the records are copied as they are, in
+// chunks of kChunk records (2 KB, `cp.async.bulk` global -> shared, completion on an mbarrier), so
+// that neither the global loads nor the shared-memory stores of the staging pass through the SM's
+// load/store pipe, which bounded this kernel while threads staged the records.  Measured on the
+// 512-profile workload: 256-byte chunks 2.37 ms, 2 KB chunks 1.99 ms, one copy per side 3.5 ms (a
+// single copy is latency-bound; a few dozen in flight per SM are not).  One slot of padding follows
+// every chunk.  What staging by threads did on the way is done by the walk instead: B's ticks are
+// moved into A's time frame when a B record is taken (A's ticks stay as stored; all tile times are
+// compared as unsigned numbers), and Eq. 2 is Phi|guards - phi_a - phi_b.
+//
+// kItems = 12 steps per thread: the lanes of a warp then start 12 path steps apart, which spreads
+// their 16-byte record reads over the bank groups better than a power of two does (16 steps and
+// 6 CTAs: 1.99 ms, 17 steps: 1.91 ms, 12 steps and 8 CTAs: 1.89 ms).
+constexpr int kPadShift = 7;
+constexpr int kChunk = 1 << kPadShift;                                  // records per bulk copy
 __device__ __forceinline__ uint32_t rec_slot(uint32_t i) { return i + (i >> kPadShift); }
 constexpr int kTileLoad = kTileItems + 2;                               // one look-ahead record per side
-constexpr int kTop = ((kTileLoad + 31) / 32) * 32 + 31;                  // unified index of B[0]; = 31 mod 32 so that
-                                                                         // a warp's descending run starts on a pad boundary
-constexpr int kRecSlots = kTop + (kTop >> kPadShift) + 2;
-constexpr int kTileCtasPerSm = 6;
-constexpr int kStageBatch = 3;                                           // global loads in flight per thread
-constexpr int kStageRounds = (kTileLoad + kTileThreads * kStageBatch - 1) / (kTileThreads * kStageBatch);
+constexpr int kTopIndex = kTileLoad + kChunk;                           // unified indices stay below this
+constexpr int kRecSlots = kTopIndex + (kTopIndex >> kPadShift) + 1;
+constexpr int kTileCtasPerSm = 8;
+constexpr unsigned long long kWaitNs = 1000000000ull;                    // bound of every wait on a copy: 1 s
+constexpr uint32_t kWaitSpins = 1u << 24;
 
 template <bool kWithV>
 __device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned long long V, uint32_t ties,
@@ -257,32 +266,60 @@ __device__ __forceinline__ float small_int_to_float(uint32_t v) {
     return __uint_as_float(0x4B000000u | v) - 8388608.0f;
 }
 
-// one side of the staging: records src[0..n) -> unified indices first, first+step, ...
-// (step = +1 for A, -1 for B); kSlack: store cap - phi instead of phi
-template <bool kSlack, int kDir>
-__device__ __forceinline__ void stage_side(const uint4* __restrict__ src, uint32_t n, uint32_t base_tick, PhiCap cap,
-                                           uint4* s_rec) {
-    // thread t handles records t, t + 128, ...; 128 is a multiple of the padding period, so the
-    // padded slot advances by a constant per trip
-    const uint32_t i0 = kDir > 0 ? threadIdx.x : (uint32_t)kTop - threadIdx.x;
-    uint4* rp = s_rec + rec_slot(i0);
-    constexpr int kRecStep = kDir * (kTileThreads + (kTileThreads >> kPadShift));
-#pragma unroll
-    for (int round = 0; round < kStageRounds; ++round) {
-        const uint32_t r0 = threadIdx.x + round * kStageBatch * kTileThreads;
-        if (r0 >= n) break;
-        uint4 r[kStageBatch];
-#pragma unroll
-        for (int j = 0; j < kStageBatch; ++j)
-            if (r0 + j * kTileThreads < n) r[j] = __ldg(src + r0 + j * kTileThreads);
-#pragma unroll
-        for (int j = 0; j < kStageBatch; ++j) {
-            if (r0 + j * kTileThreads < n) {
-                r[j].x -= base_tick; r[j].y -= base_tick;
-                if (kSlack) { r[j].z = cap.lo - r[j].z; r[j].w = cap.hi - r[j].w; }
-                rp[(round * kStageBatch + j) * kRecStep] = r[j];
-            }
-        }
+// ---- asynchronous staging: mbarrier + bulk copies ---------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+// one arrival that also announces `bytes` of copies that will complete on the barrier
+__device__ __forceinline__ void mbar_arrive_expect(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// waits for the phase with the given parity; gives up after kWaitNs (and, should the timer not
+// advance, after kWaitSpins polls)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (global_ns() - t0 > kWaitNs) return false;
+    }
+    return false;
+}
+// bytes: a multiple of 16; both addresses 16-byte aligned
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+// copies of one tile: chunk c of A goes to slots 17c.., chunk c of B to slots 17 (b_off/16 + c)..
+__device__ __forceinline__ void stage_tile_async(const uint4* __restrict__ records, const TileDesc& d, uint32_t loadA,
+                                                 uint32_t loadB, uint32_t b_off, uint4* s_rec, uint64_t* bar) {
+    const uint32_t nA = (loadA + kChunk - 1) / kChunk, nB = (loadB + kChunk - 1) / kChunk;
+    for (uint32_t c = threadIdx.x; c < nA + nB; c += kTileThreads) {
+        const bool isA = c < nA;
+        const uint32_t k = isA ? c : c - nA;
+        const uint32_t left = (isA ? loadA : loadB) - k * kChunk;
+        const uint32_t cnt = left < (uint32_t)kChunk ? left : (uint32_t)kChunk;
+        const uint4* src = records + (isA ? d.recA : d.recB) + k * kChunk;
+        uint4* dst = s_rec + (size_t)(kChunk + 1) * ((isA ? 0u : b_off / kChunk) + k);
+        bulk_copy_g2s(dst, src, cnt * (uint32_t)sizeof(uint4), bar);
     }
 }
 
@@ -296,14 +333,15 @@ __device__ __forceinline__ float fast_rcp(float x) {
 
 // one step of the walk for the pairing (ra, rb).  A step that is not live (ragged tail of a walk)
 // touches nothing: the registers may then hold a record from beyond the staged range.
+// ra holds A's record as stored, rb holds B's with its ticks moved into A's frame (+ delta).
 // fa, fb: the two kernels' resident warps as floats (o = warps / W; W cancels in o_i / (o_i + o_j)).
 // Two kernels without a resident block never interfere, so the guard of the reciprocal only keeps
 // 0 * inf out of the sums.
 #define ROOMIE_WALK_STEP(live)                                                                         \
     if (live) {                                                                                        \
-        const int32_t Ea = (int32_t)ra.y, Eb = (int32_t)rb.y;                                          \
-        const int32_t ov = min(Ea, Eb) - max((int32_t)ra.x, (int32_t)rb.x);                            \
-        const bool hit = (ov > 0) && phi_exceeds(ra.z, ra.w, rb.z, rb.w);                              \
+        const uint32_t Ea = ra.y, Eb = rb.y;                                                           \
+        const int32_t ov = (int32_t)(min(Ea, Eb) - max(ra.x, rb.x));                                   \
+        const bool hit = (ov > 0) && phi_exceeds(cap.lo - ra.z, cap.hi - ra.w, rb.z, rb.w);            \
         const float tw = (hit ? (float)ov : 0.0f) * fast_rcp(fmaxf(fa + fb, 1.0f));  /* overlap/(o_i+o_j) */ \
         di = fmaf(tw, fa, di);                                                                         \
         dj = fmaf(tw, fb, dj);                                                                         \
@@ -313,12 +351,13 @@ __device__ __forceinline__ float fast_rcp(float x) {
         /* whole warp, whichever side each lane advances                                           */  \
         const bool adv_a = Ea <= Eb;                                                                   \
         x += adv_a ? 1u : 0u;                                                                          \
-        ib -= adv_a ? 0u : 1u;                                                                         \
+        ib += adv_a ? 0u : 1u;                                                                         \
         const uint4 r = s_rec[rec_slot(adv_a ? x : ib)];                                               \
+        const float f = small_int_to_float(r.z >> kWarpShift);                                         \
         if (adv_a) {                                                                                   \
-            ra = r; fa = small_int_to_float(wconst - (r.z >> kWarpShift));                             \
+            ra = r; fa = f;                                                                            \
         } else {                                                                                       \
-            rb = r; fb = small_int_to_float(r.z >> kWarpShift);                                        \
+            rb = r; rb.x += delta; rb.y += delta; fb = f;                                              \
         }                                                                                              \
     }
 
@@ -326,39 +365,53 @@ template <bool kWithV>
 __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_kernel(TileArgs g) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint4* s_rec = reinterpret_cast<uint4*>(smem_raw);
+    __shared__ __align__(8) uint64_t s_bar;
     __shared__ float s_f[2 * kTileThreads / 32];
     __shared__ unsigned long long s_v[kTileThreads / 32];
     __shared__ uint32_t s_t[kTileThreads / 32];
 
+    if (threadIdx.x == 0) mbar_init(&s_bar, 1);
+    __syncthreads();
     const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
-    // warps field of a staged A record holds (W + guard) - warps_a
-    const uint32_t wconst = g.cap.lo >> kWarpShift;
+    const PhiCap cap = g.cap;
+    uint32_t parity = 0;
 
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
         const TileDesc d = g.tiles[t];
         const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
+        const uint32_t b_off = (loadA + kChunk - 1) & ~(uint32_t)(kChunk - 1);
+        if (threadIdx.x == 0) mbar_arrive_expect(&s_bar, (loadA + loadB) * (uint32_t)sizeof(uint4));
         __syncthreads();                                   // previous tile fully consumed
-        stage_side<true, +1>(g.records + d.recA, loadA, d.baseA, g.cap, s_rec);
-        stage_side<false, -1>(g.records + d.recB, loadB, d.baseB, g.cap, s_rec);
-        __syncthreads();
+        stage_tile_async(g.records, d, loadA, loadB, b_off, s_rec, &s_bar);
+        const bool arrived = mbar_wait_bounded(&s_bar, parity);
+        parity ^= 1u;
+        if (!__syncthreads_and(arrived)) {
+            // a copy did not arrive within the bound: report it, give the copies in flight one more
+            // bounded wait so that none lands after the CTA has gone, and stop
+            if (threadIdx.x == 0) atomicOr(g.status, ROOMIE_FLAG_WAIT_TIMEOUT);
+            if (!arrived) mbar_wait_bounded(&s_bar, parity ^ 1u);
+            return;
+        }
         const uint32_t len = d.cntA + d.cntB;
         const uint32_t diag = threadIdx.x * kItems;
+        const uint32_t delta = d.baseA - d.baseB;          // B tick + delta = the same instant in A's ticks
         float di = 0.0f, dj = 0.0f;
         unsigned long long V = 0;
         uint32_t ties = 0;
         if (diag < len) {
             // this thread's start point on the tile's merge path (A first on equal end times):
-            // B record y sits at unified index kTop - y
+            // B record y sits at unified index b_off + y
             uint32_t lo = diag > d.cntB ? diag - d.cntB : 0u, hi = diag < d.cntA ? diag : d.cntA;
-            const uint32_t btop = (uint32_t)(kTop + 1) - diag;             // index of B[diag - 1 - mid] is btop + mid
+            const uint32_t bdiag = b_off + diag - 1u;                      // index of B[diag - 1 - mid] is bdiag - mid
             while (lo < hi) {
                 const uint32_t mid = (lo + hi) >> 1;
-                if ((int32_t)s_rec[rec_slot(mid)].y <= (int32_t)s_rec[rec_slot(btop + mid)].y) lo = mid + 1;
+                if (s_rec[rec_slot(mid)].y <= s_rec[rec_slot(bdiag - mid)].y + delta) lo = mid + 1;
                 else hi = mid;
             }
-            uint32_t x = lo, ib = (uint32_t)kTop - (diag - lo);
+            uint32_t x = lo, ib = b_off + (diag - lo);
             uint4 ra = s_rec[rec_slot(x)], rb = s_rec[rec_slot(ib)];
-            float fa = small_int_to_float(wconst - (ra.z >> kWarpShift)), fb = small_int_to_float(rb.z >> kWarpShift);
+            rb.x += delta; rb.y += delta;
+            float fa = small_int_to_float(ra.z >> kWarpShift), fb = small_int_to_float(rb.z >> kWarpShift);
             if (len - diag >= (uint32_t)kItems) {
 #pragma unroll
                 for (int s = 0; s < kItems; ++s) ROOMIE_WALK_STEP(true)
@@ -700,7 +753,7 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
     TileArgs ta;
     ta.records = lv.records; ta.tiles = tiles; ta.tile_counter = counter; ta.tile_capacity = (uint32_t)need.tiles; ta.partials = partials;
     ta.inv_table = lib->share_table;
-    ta.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u; ta.cap = lv.cap;
+    ta.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u; ta.cap = lv.cap; ta.status = lib->status;
     profile_mark(st, true);
     if (pa.lockstep) {
         uint64_t grid = (uint64_t)sm_count() * 8;
@@ -784,6 +837,16 @@ extern "C" size_t roomie_pair_workspace_bytes(const roomie_library* lib, const r
     if (slots_for(lib, opts, false, 0, 0, slots) != ROOMIE_OK) return 0;
     Need need;
     batch_need(lib, opts, false, 0, 0, pair_begin, pair_end, slots, need);
+    return bytes_for(need);
+}
+
+extern "C" size_t roomie_pair_interference_workspace_bytes(const roomie_library* lib, uint32_t a, uint32_t b,
+                                                           const roomie_opts* opts) {
+    if (check_lib(lib, opts) != ROOMIE_OK || a >= lib->num_profiles || b >= lib->num_profiles) return 0;
+    uint32_t slots;
+    if (slots_for(lib, opts, true, a, b, slots) != ROOMIE_OK) return 0;
+    Need need;
+    batch_need(lib, opts, true, a, b, 0, 1, slots, need);
     return bytes_for(need);
 }
 

@@ -17,6 +17,7 @@ DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS = 2, 3, 4
 EXPORTS = [
     "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
+    "roomie_pair_interference_workspace_bytes",
     "roomie_pair_interference_static",
     "roomie_multi_estimate", "roomie_place", "roomie_place_batch", "roomie_optimal_workspace_bytes",
     "roomie_optimal_assignment", "roomie_assignment_cost", "roomie_strerror", "roomie_last_cuda_error",
@@ -44,6 +45,8 @@ def _load():
     dll.roomie_share_table_floats.restype = C.c_size_t
     dll.roomie_pair_workspace_bytes.restype = C.c_size_t
     dll.roomie_pair_workspace_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64]
+    dll.roomie_pair_interference_workspace_bytes.restype = C.c_size_t
+    dll.roomie_pair_interference_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p]
     dll.roomie_pair_matrix.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     dll.roomie_pair_interference.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
@@ -288,11 +291,7 @@ def pair_interference(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1,
     o = _opts(mode, n_align, start_filter)
     res, det = _pair_outputs(dev, detail_capacity)
     if workspace is None:
-        qa = int(lib.offsets_host[a + 1] - lib.offsets_host[a])
-        qb = int(lib.offsets_host[b + 1] - lib.offsets_host[b])
-        slots = (qa * qb) if n_align == 0 else n_align * n_align
-        tiles = slots * ((qa + qb) // 2048 + 2)
-        workspace = _workspace(4096 + slots * 16 + tiles * 64, dev)
+        workspace = _workspace(_dll.roomie_pair_interference_workspace_bytes(C.byref(lib.c), a, b, C.byref(o)), dev)
     _check(_dll.roomie_pair_interference(C.byref(lib.c), a, b, C.byref(o), _ptr(res["P2"]), _ptr(res["evals"]),
                                          C.byref(det) if det is not None else None, _ptr(workspace),
                                          workspace.numel(), _stream(stream)), "roomie_pair_interference")
