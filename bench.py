@@ -38,13 +38,29 @@ UNIT = "evals/s"
 
 
 def walk_kernel_dram_bytes(num_kernels, evals, walks):
-    """DRAM bytes (read + write) of one launch of the pairwise walk kernel.  Not measured on the full
-    workload: the ncu capture of a small case (profiles/timeline_tiles_kernel_config3.md) shows
-    compulsory first-touch reads only - 16 B per library record plus the 32 B descriptor of every tile
-    of 1536 path steps, partial results staying in L2 - and this model reproduces that capture
-    (6.52 MB against 6.57 MB measured).  Every further read of a record is served by L2."""
+    """Model of the DRAM bytes (read + write) of one launch of the pairwise walk kernel: compulsory first-touch
+    reads only - 16 B per library record plus the 32 B descriptor of every tile of 1536 path steps, partial
+    results staying in L2; every further read of a record is served by L2.  It reproduces the ncu captures of
+    configuration 3 (profiles/timeline_tiles_kernel_config3.md): 6.71 MB against 6.74 MB measured at 128
+    profiles, 38.35 MB against 38.39 MB at 512."""
     tiles = evals / 1536.0 + walks / 2.0
     return int(16 * num_kernels + 32 * tiles)
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch on the default workload (configuration 3, all 512
+# profiles, base setting), from an ncu capture of this program (profiles/timeline_tiles_kernel_config3.md)
+MEASURED_WALK_TRAFFIC = {(3, 512, "base"): 38328832 + 62720}
+
+
+def walk_kernel_traffic(args, num_kernels, evals, P):
+    if args.setting != "base":
+        return None, "not captured for this setting"
+    key = (args.config, P, args.setting)
+    if key in MEASURED_WALK_TRAFFIC:
+        return MEASURED_WALK_TRAFFIC[key], "ncu capture of this workload (profiles/timeline_tiles_kernel_config3.md)"
+    return (walk_kernel_dram_bytes(num_kernels, evals, P * (P + 1) // 2),
+            "modelled: 16 B per record + 32 B per tile, which reproduces the ncu captures of configuration 3 at 128 "
+            "and 512 profiles (profiles/timeline_tiles_kernel_config3.md)")
 
 
 def parse_args():
@@ -367,8 +383,8 @@ def main():
                          "unit": "GB/s", "frac": (achieved / peak) if achieved else None, "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": alg / launches_per_matrix if walk_launches else None,
                          "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix,
-                         "traffic": walk_kernel_dram_bytes(K, evals_per_step, P * (P + 1) // 2) if args.setting == "base" else None,
-                         "traffic_source": "modelled from the ncu small-case capture (profiles/timeline_tiles_kernel_config3.md)",
+                         "traffic": walk_kernel_traffic(args, K, evals_per_step, P)[0],
+                         "traffic_source": walk_kernel_traffic(args, K, evals_per_step, P)[1],
                          "note": "the library (16 B x K) is L2-resident: operand bytes are re-read from L2, not from HBM"},
         }
         if not args.no_cpu_baseline:
