@@ -312,7 +312,7 @@ def main():
 
     # the same cluster shape as many independent arrival streams (one CTA each): what the GPU is for on
     # this row, since a single stream is one dependent chain
-    S, nb = 8 * 148, min(2048, len(cl.arr_id))
+    S, nb = 10 * 148, min(2048, len(cl.arr_id))
     roll = (np.arange(S)[:, None] * 7 + np.arange(nb)[None, :]) % len(cl.arr_id)
     b_ids = torch.from_numpy(np.tile(cl.ids, (S, 1))).to(dev)
     b_exp = torch.from_numpy(np.tile(cl.expiry.view(np.int32), (S, 1))).to(dev)

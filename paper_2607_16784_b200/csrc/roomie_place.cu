@@ -70,6 +70,7 @@ struct PlaceArgs {
     uint32_t gpus_per_warp; // fast kernel: GPUs owned by each warp
     int admit_rule;         // 0: mean drop < lambda, 1: largest member drop < lambda
     int objective;          // 0: lowest mean drop, 1: lowest largest drop, 2: lowest drop of the arrival
+    uint32_t chunk;         // fast kernel: arrivals staged in shared memory at a time (<= kArrChunk)
 };
 
 constexpr unsigned long long kNoGpu = ~0ull;
@@ -357,9 +358,10 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
     const uint32_t oRING = 4 * GR + GR * R + gpu;         // [4][2][slot][gpu]
     const uint32_t oYOUNG = 4 * GR + GR * R + 8 * GR;     // [kYoungRing][kYoungD][2]
     const uint32_t oPUB = (oYOUNG + kYoungRing * kYoungD * 2 + 1) & ~1u;   // [G] 64-bit: order list | count << 32
-    const uint32_t oARR = oPUB + 2 * G;                   // ids [kArrChunk + 2 kLead], then lifetimes [kArrChunk]
-    const uint32_t oLIFE = oARR + kArrChunk + 2 * kLead;
-    const uint32_t oOUT = oLIFE + kArrChunk;              // decisions of the chunk: gpu, mean, mu_arr [3][kArrChunk]
+    const uint32_t chunk = g.chunk;
+    const uint32_t oARR = oPUB + 2 * G;                   // ids [chunk + 2 kLead], then lifetimes [chunk]
+    const uint32_t oLIFE = oARR + chunk + 2 * kLead;
+    const uint32_t oOUT = oLIFE + chunk;                  // decisions of the chunk: gpu, mean, mu_arr [3][chunk]
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(sm);
     volatile unsigned long long* pub = reinterpret_cast<volatile unsigned long long*>(sm + oPUB);
     __shared__ unsigned long long s_key[2][32];
@@ -420,8 +422,8 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
         }
     };
 
-    for (uint32_t k0 = 0; k0 < g.n; k0 += kArrChunk) {
-        const uint32_t kn = min(kArrChunk, g.n - k0);
+    for (uint32_t k0 = 0; k0 < g.n; k0 += chunk) {
+        const uint32_t kn = min(chunk, g.n - k0);
         // stage arrival ids [k0 - kLead, k0 + kn + kLead) and lifetimes [k0, k0 + kn)
         __syncthreads();
         for (uint32_t i = tid; i < kn + 2 * kLead; i += blockDim.x) {
@@ -503,7 +505,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             // results stay in shared memory until the chunk ends: a global store inside the loop would
             // have to complete before every barrier
             if (best == kNoGpu) {
-                if (tid == 0) { smi[oOUT + k] = -1; sm[oOUT + kArrChunk + k] = 0.0f; sm[oOUT + 2 * kArrChunk + k] = 0.0f; }
+                if (tid == 0) { smi[oOUT + k] = -1; sm[oOUT + chunk + k] = 0.0f; sm[oOUT + 2 * chunk + k] = 0.0f; }
             } else if (owner && gpu == (uint32_t)(best & 0xffffffffu)) {
                 const uint32_t pn = __ffs(free_mask) - 1u;                   // lowest free physical slot
                 free_mask &= ~(1u << pn);
@@ -530,15 +532,15 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 __threadfence_block();                                       // id before the list that names its slot
                 pub[gpu] = (unsigned long long)ord | ((unsigned long long)c << 32);
                 smi[oOUT + k] = (int32_t)gpu;
-                sm[oOUT + kArrChunk + k] = mean;
-                sm[oOUT + 2 * kArrChunk + k] = mu_inc;
+                sm[oOUT + chunk + k] = mean;
+                sm[oOUT + 2 * chunk + k] = mu_inc;
             }
         }
         __syncthreads();
         for (uint32_t i = tid; i < kn; i += blockDim.x) {
             g.gpu_out[k0 + i] = smi[oOUT + i];
-            if (g.mean_out) g.mean_out[k0 + i] = sm[oOUT + kArrChunk + i];
-            if (g.mu_arr_out) g.mu_arr_out[k0 + i] = sm[oOUT + 2 * kArrChunk + i];
+            if (g.mean_out) g.mean_out[k0 + i] = sm[oOUT + chunk + i];
+            if (g.mu_arr_out) g.mu_arr_out[k0 + i] = sm[oOUT + 2 * chunk + i];
         }
     }
     cp_async_wait<0>();
@@ -590,8 +592,10 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t GR = (size_t)a.G * a.R;
+    // many independent streams: a short staging chunk keeps the CTA small enough for 5 per SM
+    a.chunk = num_streams > 1 ? 128u : kArrChunk;
     const size_t fast_bytes = GR * 4 * 4 + GR * a.R * 4 + 4 * 2 * GR * 4 + (kYoungRing * kYoungD * 2 + 2) * 4 +
-                              2 * a.G * 4 + (5 * kArrChunk + 2 * kLead) * sizeof(int32_t);
+                              2 * a.G * 4 + (5 * a.chunk + 2 * kLead) * sizeof(int32_t);
     if (a.R <= 8 && a.G <= 512 && fast_bytes <= 160 * 1024) {
         // up to 8 slots per GPU: matrix elements are fetched three arrivals ahead by fetch warps
         a.matrix_mode = 1; a.pair_cache = 1;
