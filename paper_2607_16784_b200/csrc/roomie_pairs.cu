@@ -709,6 +709,8 @@ static int check_lib(const roomie_library* lib, const roomie_opts* o) {
     if (!lib || !o || !lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->share_table ||
         !lib->status || lib->num_profiles == 0)
         return ROOMIE_ERR_INVALID_ARG;
+    // 16-byte loads and bulk copies of the records: a misaligned table would fault on the device
+    if (reinterpret_cast<uintptr_t>(lib->records) & 15u) return ROOMIE_ERR_INVALID_ARG;
     if (o->walk_mode < ROOMIE_WALK_TIMELINE || o->walk_mode > ROOMIE_WALK_DETAILED_FCFS) return ROOMIE_ERR_INVALID_ARG;
     return validate_spec(&lib->spec);
 }

@@ -40,3 +40,47 @@ def test_host_side_argument_checks():
     dll.roomie_share_table_floats.restype = ctypes.c_size_t
     assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 65536, 164 * 1024, 2048, 32))) == 2 * 64 + 1
     assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 1 << 18, 164 * 1024, 2048, 32))) == 0   # RANGE
+
+
+def test_workspace_size_queries_are_host_only():
+    """The two size queries read only the host copy of the profile offsets: they answer without a GPU, agree with
+    each other on a single pair, grow with the alignment count and refuse a record table that is not 16-byte aligned."""
+    import numpy as np
+    import paper_2607_16784_b200 as pkg
+    from paper_2607_16784_b200 import roomie as rm
+    dll = ctypes.CDLL(pkg.lib_path())
+    dll.roomie_pair_workspace_bytes.restype = ctypes.c_size_t
+    dll.roomie_pair_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64]
+    dll.roomie_pair_interference_workspace_bytes.restype = ctypes.c_size_t
+    dll.roomie_pair_interference_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
+                                                             ctypes.c_void_p]
+    offsets = np.array([0, 5000, 5003, 9000], np.uint32)
+    fake = 0x10000                                           # never dereferenced by the size queries
+
+    def library(records_ptr):
+        return rm._Library(3, 9000, offsets.ctypes.data, fake, records_ptr, fake, fake, fake,
+                           rm._Spec(108, 65536, 164 * 1024, 2048, 32))
+
+    def opts(mode, n_align):
+        return rm._Opts(mode, n_align, 0, 0.5, 8, 0, 0)
+
+    lib = library(fake)
+    one = dll.roomie_pair_interference_workspace_bytes(ctypes.byref(lib), 0, 2, ctypes.byref(opts(0, 1)))
+    many = dll.roomie_pair_interference_workspace_bytes(ctypes.byref(lib), 0, 2, ctypes.byref(opts(0, 8)))
+    assert 0 < one < many
+    # pair (0, 2) is pair index 2 of the upper triangle (0,0), (0,1), (0,2), (1,1), ...
+    assert dll.roomie_pair_workspace_bytes(ctypes.byref(lib), ctypes.byref(opts(0, 1)), 2, 3) == one
+    whole = dll.roomie_pair_workspace_bytes(ctypes.byref(lib), ctypes.byref(opts(0, 1)), 0, 6)
+    assert whole > one
+    assert dll.roomie_pair_workspace_bytes(ctypes.byref(lib), ctypes.byref(opts(0, 1)), 4, 4) == 0       # empty range
+    assert dll.roomie_pair_interference_workspace_bytes(ctypes.byref(lib), 0, 3, ctypes.byref(opts(0, 1))) == 0
+    assert dll.roomie_pair_interference_workspace_bytes(ctypes.byref(lib), 0, 2, ctypes.byref(opts(9, 1))) == 0
+    # the full Cartesian product of a 5000 x 3997 pair is beyond the 4096 alignments a pair may have
+    assert dll.roomie_pair_interference_workspace_bytes(ctypes.byref(lib), 0, 2, ctypes.byref(opts(0, 0))) == 0
+    bad = library(fake + 8)
+    assert dll.roomie_pair_interference_workspace_bytes(ctypes.byref(bad), 0, 2, ctypes.byref(opts(0, 1))) == 0
+    dll.roomie_pair_matrix.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint64,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t,
+                                       ctypes.c_void_p]
+    assert dll.roomie_pair_matrix(ctypes.byref(bad), ctypes.byref(opts(0, 1)), 0, 6, fake, None, fake * 16, 1 << 20,
+                                  None) == -1                # INVALID_ARG before any CUDA call
