@@ -66,8 +66,8 @@ def walk_kernel_traffic(args, num_kernels, evals, P):
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="roomie", choices=["roomie", "reference"])
     ap.add_argument("--config", type=int, default=3, help="library configuration (0-4)")
     ap.add_argument("--setting", default="base", choices=["base", "greedy", "lockstep_full", "detailed"],
