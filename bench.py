@@ -348,17 +348,18 @@ def main():
         launches_per_matrix = walk_launches / args.steps
         achieved = alg / launches_per_matrix / (per_launch_ms * 1e-3) / 1e9 if walk_launches else None
         if args.setting == "lockstep_full":
-            # compute-bound kernel: table cells visited (q_a*q_b per pair, at most 4 passes of the exact
-            # median) against the plain-ALU issue peak, 148 SMs x 128 lanes x SM clock, divided by the 54
-            # lane-instructions one cell visit takes (profiles/lockstep_full_kernel_config2.md)
+            # compute-bound kernel: table cells visited (q_a*q_b per pair and pass; the exact median takes 3
+            # passes, 4 when the number of kept alignments is even: 3 are counted) against the plain-ALU issue
+            # peak, 148 SMs x 128 lanes x SM clock, divided by the 53 lane-instructions one cell visit takes
+            # (profiles/lockstep_full_kernel_config2.md)
             q = lib.q().astype(np.int64)
             ia, ib = np.triu_indices(P)
-            visits = 4.0 * float((q[ia] * q[ib]).sum())
-            peak_visits = 148 * 128 * 1.965e9 / 54.0 / 1e9
+            visits = 3.0 * float((q[ia] * q[ib]).sum())
+            peak_visits = 148 * 128 * 1.965e9 / 53.0 / 1e9
             ach = visits / (per_launch_ms * 1e-3) / 1e9 if walk_launches else None
             roofline = {"bound": "alu", "kernel": "lockstep_full_kernel", "achieved": ach, "peak": peak_visits,
                         "unit": "G cell visits/s", "frac": (ach / peak_visits) if ach else None,
-                        "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz / 54 lane-instructions per visit",
+                        "peak_source": "derived: 148 SMs x 128 lanes x 1.965 GHz / 53 lane-instructions per visit",
                         "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix, "traffic": None}
         else:
             roofline = None

@@ -5,8 +5,8 @@
 // The delay of alignment (s_i, s_j) is the sum of the charged terms along the diagonal that starts
 // at (s_i, s_j):  delta_i(s_i, s_j) = sum_t hit(s_i+t, s_j+t) * d_{s_i+t} * o_i/(o_i+o_j), so all
 // q_i*q_j alignments of a pair are the suffix sums along the q_i+q_j-1 diagonals of one q_i x q_j
-// table: q_i*q_j work instead of q_i*q_j*min(q).  The table is never stored: one thread walks one
-// diagonal from its far end (coalesced record loads across neighbouring diagonals) and the values go
+// table: q_i*q_j work instead of q_i*q_j*min(q).  The table is never stored: one thread walks four
+// neighbouring diagonals from their far ends and the values go
 // straight into the histogram of an exact radix select (3 digit passes of 11/11/10 bits over the
 // float bits, which order like the non-negative values - the first one also counts the kept
 // alignments - plus, for an even count, a pass for the upper middle value).  Every pass recomputes the suffix sums; a suffix sum is accumulated in double
@@ -38,31 +38,69 @@ struct FullSelect {               // state of the radix select of one direction
 };
 
 // walks every diagonal of the pair once; `visit(vi_bits, vj_bits, walk_len)` is called for every
-// kept alignment with the float bits of its two delays and the length of its walk
+// kept alignment with the float bits of its two delays and the length of its walk.
+// One thread takes kDiags neighbouring diagonals at a time and moves up the table row by row: row i
+// pairs A[i] with B[i - off - m], m = 0..kDiags-1, and the next row needs only one new record of each
+// profile (the B records slide along a register window), so a cell costs half a record load and the
+// per-record conversions (duration * warps as float) are done once per record, not once per cell.
+constexpr int kDiags = 4;
+
+struct FullRec {                  // what a cell needs of one kernel
+    uint32_t lo, hi;              // packed demand
+    uint32_t w;                   // resident warps
+    float x;                      // duration in ticks * warps
+};
+
+__device__ __forceinline__ FullRec full_rec(const uint4& r) {
+    FullRec f;
+    f.lo = r.z; f.hi = r.w;
+    f.w = r.z >> kWarpShift;
+    f.x = (float)(r.y - r.x) * small_int_to_float(f.w);
+    return f;
+}
+
 template <class Visit>
 __device__ __forceinline__ void full_walk(const uint4* __restrict__ A, const uint4* __restrict__ B, uint32_t na,
                                           uint32_t nb, PhiCap cap, const float* s_inv, int start_filter,
                                           Visit visit) {
-    const uint32_t n_diag = na + nb - 1;
-    for (uint32_t dg = threadIdx.x; dg < n_diag; dg += kFullThreads) {
-        // diagonal dg holds the cells (i, j) with i - j = dg - (nb - 1); walk it from its far end
-        const int32_t off = (int32_t)dg - (int32_t)(nb - 1);
-        const uint32_t i_lo = off > 0 ? (uint32_t)off : 0u;
-        const uint32_t i_hi = min(na - 1, (uint32_t)((int32_t)(nb - 1) + off));       // inclusive
-        double si = 0.0, sj = 0.0;
-        uint32_t len = 0;
-        for (uint32_t i = i_hi + 1; i-- > i_lo;) {
-            const uint32_t j = (uint32_t)((int32_t)i - off);
-            const uint4 ra = __ldg(&A[i]), rb = __ldg(&B[j]);
-            ++len;
-            const bool hit = phi_exceeds(cap.lo - ra.z, cap.hi - ra.w, rb.z, rb.w);
-            if (hit) {
-                const uint32_t wa = ra.z >> kWarpShift, wb = rb.z >> kWarpShift;
-                const float inv = s_inv[wa + wb];
-                si += (double)(((float)(ra.y - ra.x) * inv) * small_int_to_float(wa));
-                sj += (double)(((float)(rb.y - rb.x) * inv) * small_int_to_float(wb));
+    const int32_t n_diag = (int32_t)(na + nb - 1);
+    const int32_t n_groups = (n_diag + kDiags - 1) / kDiags;
+    const int32_t last_a = (int32_t)na - 1, last_b = (int32_t)nb - 1;
+    for (int32_t grp = (int32_t)threadIdx.x; grp < n_groups; grp += kFullThreads) {
+        // diagonal m of the group holds the cells (i, j) with i - j = off + m
+        const int32_t off = grp * kDiags - last_b;
+        const int32_t i_top = min(last_a, last_b + off + kDiags - 1);      // highest row any of them reaches
+        const int32_t i_bot = max(0, off);                                  // lowest row any of them reaches
+        double si[kDiags], sj[kDiags];
+        uint32_t len[kDiags];
+        FullRec rb[kDiags];
+#pragma unroll
+        for (int m = 0; m < kDiags; ++m) {
+            si[m] = 0.0; sj[m] = 0.0; len[m] = 0;
+            const int32_t j = i_top - off - m;
+            rb[m] = full_rec(__ldg(&B[min(max(j, 0), last_b)]));             // out-of-range cells are skipped below
+        }
+        for (int32_t i = i_top; i >= i_bot; --i) {
+            const FullRec ra = full_rec(__ldg(&A[i]));
+#pragma unroll
+            for (int m = 0; m < kDiags; ++m) {
+                const int32_t j = i - off - m;
+                if (j >= 0 && j <= last_b) {                               // cell (i, j) exists (j < 0 also ends short groups)
+                    ++len[m];
+                    const bool hit = phi_exceeds(cap.lo - ra.lo, cap.hi - ra.hi, rb[m].lo, rb[m].hi);
+                    if (hit) {
+                        const float inv = s_inv[ra.w + rb[m].w];
+                        si[m] += (double)(ra.x * inv);
+                        sj[m] += (double)(rb[m].x * inv);
+                    }
+                    if (!start_filter || hit) visit(__float_as_uint((float)si[m]), __float_as_uint((float)sj[m]), len[m]);
+                }
             }
-            if (!start_filter || hit) visit(__float_as_uint((float)si), __float_as_uint((float)sj), len);
+            // next row: diagonal m meets the record diagonal m + 1 met in this row
+#pragma unroll
+            for (int m = 0; m + 1 < kDiags; ++m) rb[m] = rb[m + 1];
+            const int32_t jn = i - 1 - off - (kDiags - 1);
+            rb[kDiags - 1] = full_rec(__ldg(&B[min(max(jn, 0), last_b)]));
         }
     }
 }
