@@ -13,6 +13,7 @@
 //             path search + kItems sequential steps, warp-shuffle reduction -> one partial
 //   finalize  one CTA per pair: sum partials per alignment, median over alignments, gamma, /T
 #include "roomie_common.cuh"
+#include <vector>
 
 namespace roomie {
 
@@ -624,27 +625,52 @@ static uint32_t host_grid_count(uint32_t q, uint32_t A) { return (A == 0 || A > 
 struct Need { uint64_t walks, tiles; };
 
 // upper bound of walk slots and tiles for pairs [p0, p1): a walk of a pair has at most
-// q_a + q_b - 1 steps whatever its alignment
+// q_a + q_b - 1 steps whatever its alignment.  Short ranges are counted pair by pair; long ones row by
+// row from prefix sums over the profiles (a matrix of 131 328 pairs would otherwise keep the GPU waiting
+// for 0.1 ms of host arithmetic in every call), rounding each row up, i.e. by less than one tile per walk.
 static bool batch_need(const roomie_library* lib, const roomie_opts* o, bool explicit_pair, uint32_t ea, uint32_t eb,
                        uint64_t p0, uint64_t p1, uint32_t slots, Need& need) {
     const uint32_t* off = lib->offsets_host;
+    const uint32_t P = lib->num_profiles;
+    const bool detailed = o->walk_mode >= ROOMIE_WALK_DETAILED_EQUAL, lockstep = o->walk_mode == ROOMIE_WALK_LOCKSTEP;
     uint64_t tiles = 0;
     auto add = [&](uint32_t a, uint32_t b) {
         const uint32_t qa = off[a + 1] - off[a], qb = off[b + 1] - off[b];
         const uint64_t n = (uint64_t)host_grid_count(qa, o->n_align) * host_grid_count(qb, o->n_align);
-        const uint64_t per = o->walk_mode >= ROOMIE_WALK_DETAILED_EQUAL ? 1   // one result record per walk
-                             : o->walk_mode == ROOMIE_WALK_LOCKSTEP
-                                 ? ((uint64_t)(qa < qb ? qa : qb) + kTileItems - 1) / kTileItems
-                                 : ((uint64_t)qa + qb - 1 + kTileItems - 1) / kTileItems;
+        const uint64_t per = detailed ? 1                                  // one result record per walk
+                             : lockstep ? ((uint64_t)(qa < qb ? qa : qb) + kTileItems - 1) / kTileItems
+                                        : ((uint64_t)qa + qb - 1 + kTileItems - 1) / kTileItems;
         tiles += n * per;
     };
     if (explicit_pair) add(ea, eb);
-    else {
+    else if (p1 - p0 <= 64) {
         uint32_t a, b;
-        pair_of_host(p0, lib->num_profiles, a, b);
+        pair_of_host(p0, P, a, b);
         for (uint64_t p = p0; p < p1; ++p) {
             add(a, b);
-            if (++b == lib->num_profiles) { ++a; b = a; }
+            if (++b == P) { ++a; b = a; }
+        }
+    } else {
+        // G1[b] = sum of alignment starts g of the profiles before b, G2[b] = sum of g * q
+        static thread_local std::vector<uint64_t> G1, G2;
+        G1.assign((size_t)P + 1, 0); G2.assign((size_t)P + 1, 0);
+        for (uint32_t b = 0; b < P; ++b) {
+            const uint64_t q = off[b + 1] - off[b], g = host_grid_count((uint32_t)q, o->n_align);
+            G1[b + 1] = G1[b] + g;
+            G2[b + 1] = G2[b] + g * q;
+        }
+        uint32_t a, b;
+        pair_of_host(p0, P, a, b);
+        for (uint64_t left = p1 - p0; left > 0;) {
+            const uint64_t cnt = left < (uint64_t)(P - b) ? left : (uint64_t)(P - b);      // pairs (a, b .. b + cnt)
+            const uint64_t qa = off[a + 1] - off[a], ga = host_grid_count((uint32_t)qa, o->n_align);
+            const uint64_t sg = G1[b + cnt] - G1[b], sgq = G2[b + cnt] - G2[b];
+            uint64_t row;                                                  // sum over the row of g_b * tiles per walk
+            if (detailed) row = sg;
+            else if (lockstep) row = ((sgq < qa * sg ? sgq : qa * sg) + sg * (kTileItems - 1)) / kTileItems + 1;   // min(q_a, q_b) <= q_a, q_b
+            else row = (sgq + sg * (qa + kTileItems - 2)) / kTileItems + 1;
+            tiles += ga * row;
+            left -= cnt; ++a; b = a;
         }
     }
     need.walks = (explicit_pair ? 1 : (p1 - p0)) * (uint64_t)slots;
