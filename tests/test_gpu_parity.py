@@ -594,3 +594,32 @@ def test_very_long_profiles_and_single_profile_library(rm, oracle):
     got, ev = rm.pair_matrix(gl1, mode=0, n_align=8, start_filter=1)
     assert got.shape == (1, 1) and int(ev.item()) == wev
     assert_close(got.cpu().numpy(), want)
+
+
+def test_timelines_close_to_the_tick_limit(rm, oracle):
+    """Profiles whose timelines end just below 2^31 ticks (2.1 s): late alignments shift one model's ticks by up
+    to that much against the other's, so the walk's tile-local times use the whole 32-bit range."""
+    from types import SimpleNamespace
+    base = rs.make_library(3, num_profiles=4)
+    n = [1800, 2500, 900]
+    off = np.concatenate([[0], np.cumsum(n)]).astype(np.uint32)
+    K = int(off[-1])
+    rng = np.random.default_rng(5)
+    dur = np.empty(K, np.float32)
+    for p in range(3):                                            # mean duration so that T is about 2.1e9 ns
+        mean_us = 2.2e6 / n[p]
+        dur[off[p]:off[p + 1]] = (rng.uniform(0.2, 1.7, n[p]) * mean_us).astype(np.float32)
+    gap = (rng.uniform(0.0, 20.0, K)).astype(np.float32)
+    lib = SimpleNamespace(spec=base.spec, offsets=off, dur_us=dur, gap_us=gap,
+                          **{k: getattr(base, k)[:K] for k in ("grid_blocks", "block_threads", "regs_per_thread",
+                                                               "smem_per_block")})
+    ol, gl = build_both(rm, oracle, lib)
+    assert gl.status_flags() == 0 and ol.T.max() > 2.0e9
+    for kw in (dict(mode=0, n_align=1, start_filter=0), dict(mode=0, n_align=8, start_filter=0),
+               dict(mode=0, n_align=8, start_filter=1), dict(mode=1, n_align=8, start_filter=0)):
+        want, wev = oracle.pair_matrix(ol, **kw)
+        got, ev = rm.pair_matrix(gl, **kw)
+        assert int(ev.item()) == wev
+        assert_close(got.cpu().numpy(), want)
+    for a, b in ((0, 1), (2, 1)):
+        check_pair_detail(rm, oracle, ol, gl, a, b, mode=0, n_align=8, start_filter=0)
