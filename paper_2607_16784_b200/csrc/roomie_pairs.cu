@@ -224,8 +224,10 @@ struct TileArgs {
 // 512-profile workload: 256-byte chunks 2.37 ms, 2 KB chunks 1.99 ms, one copy per side 3.5 ms (a
 // single copy is latency-bound; a few dozen in flight per SM are not).  One slot of padding follows
 // every chunk.  What staging by threads did on the way is done by the walk instead: B's ticks are
-// moved into A's time frame when a B record is taken (A's ticks stay as stored; all tile times are
-// compared as unsigned numbers), and Eq. 2 is Phi|guards - phi_a - phi_b.
+// moved into A's time frame when a B record is taken (A's ticks stay as stored), and Eq. 2 is
+// Phi|guards - phi_a - phi_b.  Timelines end below 2^31 ticks, so a B tick in A's frame stays below 2^32:
+// times are compared as unsigned numbers, and since all times of one walk lie within 2^31 ticks of each
+// other an overlap is the signed difference of two of them.
 //
 // kItems = 12 steps per thread: the lanes of a warp then start 12 path steps apart, which spreads
 // their 16-byte record reads over the bank groups better than a power of two does (16 steps and
