@@ -326,6 +326,11 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
 //   - a resident placed fewer than 5 arrivals ago may have been missed by those fetches (they
 //     were issued before, or while, it was placed); its terms depend only on the arrival stream
 //     (P[arr_{j-d}][arr_j] and the transpose, d = 1..4) and are fetched on the same schedule.
+//   - the what-if loop of an owner lane is a two-stage software pipeline over its residents (the reads
+//     for resident t + 1 and t + 2 are in flight while t is summed), and it leaves behind everything
+//     the winner's update needs: the new partial sums go into a second copy of the partial-sum array
+//     (the winner only switches copies) and the resident-arrival terms into the row and column of the
+//     free slot the arrival would take, so the update itself has no loop.
 // The owners' critical path per arrival is shared-memory reads, 2c+2 float adds, one division,
 // two redux steps and one barrier; no global memory access and no copy wait.
 // ---------------------------------------------------------------------------------------
@@ -362,6 +367,9 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
     const uint32_t oARR = oPUB + 2 * G;                   // ids [chunk + 2 kLead], then lifetimes [chunk]
     const uint32_t oLIFE = oARR + chunk + 2 * kLead;
     const uint32_t oOUT = oLIFE + chunk;                  // decisions of the chunk: gpu, mean, mu_arr [3][chunk]
+    // cached partial sums, twice: every what-if writes the sums its GPU would have after taking the arrival
+    // into the other copy, and the winner just switches copies
+    uint32_t pa_cur = oPA, pa_alt = oOUT + 3 * chunk + gpu;
     const uint32_t sm_base = (uint32_t)__cvta_generic_to_shared(sm);
     volatile unsigned long long* pub = reinterpret_cast<volatile unsigned long long*>(sm + oPUB);
     __shared__ unsigned long long s_key[2][32];
@@ -389,7 +397,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             float s = 0.0f;
             for (uint32_t q = 0; q < c; ++q)
                 if (q != p) s = __fadd_rn(s, sm[oPT + (p * R + q) * G]);
-            sm[oPA + p * G] = s;
+            sm[pa_cur + p * G] = s;
         }
         pub[gpu] = (unsigned long long)ord | ((unsigned long long)c << 32);
     }
@@ -467,7 +475,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                     float s = 0.0f;
                     for (uint32_t u = 0; u < c; ++u)
                         if (u != t) s = __fadd_rn(s, sm[oPT + (p * R + ((ord >> (4 * u)) & 15u)) * G]);
-                    sm[oPA + p * G] = s;
+                    sm[pa_cur + p * G] = s;
                 }
             }
             // terms of arrival kg: ring (by physical slot) or, for young residents, arrival-to-arrival
@@ -477,17 +485,40 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             float mean = 0.0f, mu_inc = 0.0f;
             if (owner && c < R) {                                            // what-if: residents + the arrival
                 float tot = 0.0f, worst = 0.0f;
-                for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {
-                    const uint32_t p = o & 15u;
-                    const uint32_t d1 = (uint32_t)((int32_t)kg - smi[oBI + p * G]);   // arrivals since placed, minus 1 (huge if old)
-                    const bool young = d1 < (uint32_t)kYoungD;
-                    const uint32_t i0 = young ? young_k + 2 * d1 : ring_k + p * G;
-                    const float to = sm[i0];                                  // P[id][inc]
-                    const float from = sm[i0 + (young ? 1u : GR)];            // P[inc][id]
-                    const float mu_t = __fadd_rn(sm[oPA + p * G], to);
+                // two-stage pipeline over the residents: while resident t is summed, the terms of t + 1 are on
+                // their way and the birth index and cached partial sum of t + 2 are being read (past the end
+                // of the list the nibbles are 0: slot 0 is read, a valid address, and the value is dropped)
+                const uint32_t pn = __ffs(free_mask) - 1u;                   // lowest free physical slot: the arrival's, if it comes here
+                const uint32_t pt_col = oPT + pn * G, pt_row = oPT + pn * R * G;
+                uint32_t o = ord, p = o & 15u, p_c = p;
+                uint32_t d1 = (uint32_t)((int32_t)kg - smi[oBI + p * G]);    // arrivals since placed, minus 1 (huge if old)
+                bool young = d1 < (uint32_t)kYoungD;
+                uint32_t i0 = young ? young_k + 2 * d1 : ring_k + p * G;
+                float pa = sm[pa_cur + p * G];
+                float to = sm[i0];                                            // P[id][inc]
+                float from = sm[i0 + (young ? 1u : GR)];                      // P[inc][id]
+                o >>= 4; p = o & 15u;
+                int32_t bi_n = smi[oBI + p * G];
+                float pa_n = sm[pa_cur + p * G];
+                for (uint32_t t = 0; t < c; ++t) {
+                    const uint32_t p_n = p;
+                    d1 = (uint32_t)((int32_t)kg - bi_n);
+                    young = d1 < (uint32_t)kYoungD;
+                    i0 = young ? young_k + 2 * d1 : ring_k + p * G;
+                    const float to_n = sm[i0], from_n = sm[i0 + (young ? 1u : GR)], pa_c = pa_n;
+                    o >>= 4; p = o & 15u;
+                    bi_n = smi[oBI + p * G];
+                    pa_n = sm[pa_cur + p * G];
+                    const float mu_t = __fadd_rn(pa, to);
                     worst = fmaxf(worst, mu_t);
                     tot = __fadd_rn(tot, mu_t);
                     mu_inc = __fadd_rn(mu_inc, from);
+                    // what the winner will need: the new partial sum and the two terms between the
+                    // resident and the arrival (the free slot's row and column hold nothing yet)
+                    sm[pa_alt + p_c * G] = mu_t;
+                    sm[pt_col + p_c * R * G] = to;
+                    sm[pt_row + p_c * G] = from;
+                    pa = pa_c; to = to_n; from = from_n; p_c = p_n;
                 }
                 tot = __fadd_rn(tot, mu_inc);
                 mean = __fdiv_rn(tot, (float)(c + 1));
@@ -507,20 +538,11 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             if (best == kNoGpu) {
                 if (tid == 0) { smi[oOUT + k] = -1; sm[oOUT + chunk + k] = 0.0f; sm[oOUT + 2 * chunk + k] = 0.0f; }
             } else if (owner && gpu == (uint32_t)(best & 0xffffffffu)) {
-                const uint32_t pn = __ffs(free_mask) - 1u;                   // lowest free physical slot
+                const uint32_t pn = __ffs(free_mask) - 1u;                   // the slot the what-if wrote for
                 free_mask &= ~(1u << pn);
-                for (uint32_t t = 0, o = ord; t < c; ++t, o >>= 4) {         // the what-if sums become the cached ones
-                    const uint32_t p = o & 15u;
-                    const uint32_t d1 = (uint32_t)((int32_t)kg - smi[oBI + p * G]);
-                    const bool young = d1 < (uint32_t)kYoungD;
-                    const uint32_t i0 = young ? young_k + 2 * d1 : ring_k + p * G;
-                    const float to = sm[i0], from = sm[i0 + (young ? 1u : GR)];
-                    sm[oPA + p * G] = __fadd_rn(sm[oPA + p * G], to);
-                    sm[oPT + (p * R + pn) * G] = to;
-                    sm[oPT + (pn * R + p) * G] = from;
-                }
+                { const uint32_t sw = pa_cur; pa_cur = pa_alt; pa_alt = sw; } // the what-if sums become the cached ones
                 sm[oPT + (pn * R + pn) * G] = 0.0f;
-                sm[oPA + pn * G] = mu_inc;
+                sm[pa_cur + pn * G] = mu_inc;
                 smi[oID + pn * G] = smi[oARR + kl];
                 const uint32_t life = (uint32_t)smi[oLIFE + k];
                 const uint32_t e = life ? now + life : 0u;
@@ -592,9 +614,9 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t GR = (size_t)a.G * a.R;
-    // many independent streams: a short staging chunk keeps the CTA small enough for 5 per SM
-    a.chunk = num_streams > 1 ? 128u : kArrChunk;
-    const size_t fast_bytes = GR * 4 * 4 + GR * a.R * 4 + 4 * 2 * GR * 4 + (kYoungRing * kYoungD * 2 + 2) * 4 +
+    // many independent streams: a short staging chunk keeps the CTA small enough (44.4 KB) for 5 per SM
+    a.chunk = num_streams > 1 ? 32u : kArrChunk;
+    const size_t fast_bytes = GR * 5 * 4 + GR * a.R * 4 + 4 * 2 * GR * 4 + (kYoungRing * kYoungD * 2 + 2) * 4 +
                               2 * a.G * 4 + (5 * a.chunk + 2 * kLead) * sizeof(int32_t);
     if (a.R <= 8 && a.G <= 512 && fast_bytes <= 160 * 1024) {
         // up to 8 slots per GPU: matrix elements are fetched three arrivals ahead by fetch warps
