@@ -334,6 +334,17 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
 // The owners' critical path per arrival is shared-memory reads, 2c+2 float adds, one division,
 // two redux steps and one barrier; no global memory access and no copy wait.
 // ---------------------------------------------------------------------------------------
+// a / n for 1 <= n <= 9, correctly rounded like the float32 division it replaces (IEEE division is a
+// subroutine of a few dozen dependent instructions; this is a conversion, a product and a conversion).
+// The double product of a and the double nearest to 1/n is within 2^-52 (relative) of a/n.  A 24-bit a
+// divided by n <= 9 is either a float itself or at least 2^-29 (relative) away from every midpoint
+// between two neighbouring floats (the distance is a non-zero multiple of half a unit in the last place
+// divided by n), so rounding the product to float32 rounds the quotient.
+__constant__ double kInvSmall[10] = {0.0, 1.0, 1.0 / 2, 1.0 / 3, 1.0 / 4, 1.0 / 5, 1.0 / 6, 1.0 / 7, 1.0 / 8, 1.0 / 9};
+__device__ __forceinline__ float div_small(float a, uint32_t n) {
+    return __double2float_rn(__dmul_rn((double)a, kInvSmall[n]));
+}
+
 constexpr int kAhead = 3;                     // arrivals fetched ahead
 constexpr int kYoungD = kAhead + 1;           // residents this young read the arrival-to-arrival terms
 constexpr int kYoungRing = 8;                 // ring depth of the arrival-to-arrival terms
@@ -521,7 +532,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                     pa = pa_c; to = to_n; from = from_n; p_c = p_n;
                 }
                 tot = __fadd_rn(tot, mu_inc);
-                mean = __fdiv_rn(tot, (float)(c + 1));
+                mean = div_small(tot, c + 1);                                // c + 1 <= 9 in this kernel
                 key_hi = decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
             }
             const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
