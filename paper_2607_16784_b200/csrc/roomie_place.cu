@@ -535,14 +535,22 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 mean = div_small(tot, c + 1);                                // c + 1 <= 9 in this kernel
                 key_hi = decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
             }
+            // warp argmin: lowest key, then the lowest lane (= lowest GPU index of this warp) that holds it
             const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
-            const uint32_t best_lo = __reduce_min_sync(0xffffffffu, (key_hi == best_hi && key_hi != 0xffffffffu) ? gpu : 0xffffffffu);
+            const uint32_t holders = __ballot_sync(0xffffffffu, key_hi == best_hi);
+            const uint32_t best_lo = best_hi != 0xffffffffu ? (wid << 5) + (uint32_t)__ffs(holders) - 1u : 0xffffffffu;
             if (lane == 0) s_key[k & 1][wid] = ((unsigned long long)best_hi << 32) | best_lo;
             __syncthreads();
-            unsigned long long best = s_key[k & 1][0];
-            for (uint32_t w = 1; w < n_owner_warps; ++w) {
-                const unsigned long long o = s_key[k & 1][w];
-                best = o < best ? o : best;
+            unsigned long long best;
+            if (n_owner_warps == 2) {                                        // the common shape: both keys at once
+                const unsigned long long k0w = s_key[k & 1][0], k1w = s_key[k & 1][1];
+                best = k1w < k0w ? k1w : k0w;
+            } else {
+                best = s_key[k & 1][0];
+                for (uint32_t w = 1; w < n_owner_warps; ++w) {
+                    const unsigned long long o = s_key[k & 1][w];
+                    best = o < best ? o : best;
+                }
             }
             // results stay in shared memory until the chunk ends: a global store inside the loop would
             // have to complete before every barrier
