@@ -355,6 +355,9 @@ __device__ __forceinline__ void cp_async_4_s(uint32_t smem_addr, const void* gme
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"(smem_addr), "l"(gmem_src) : "memory");
 }
 
+// kPlain: Algorithm 2 as printed (admit on the mean drop, choose the lowest mean drop); the rule and the
+// objective are then compile-time facts and the largest member drop is not tracked
+template <bool kPlain>
 __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
     select_stream(g);
     // one float/int array; every region is addressed by a 32-bit word index
@@ -521,7 +524,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                     bi_n = smi[oBI + p * G];
                     pa_n = sm[pa_cur + p * G];
                     const float mu_t = __fadd_rn(pa, to);
-                    worst = fmaxf(worst, mu_t);
+                    if (!kPlain) worst = fmaxf(worst, mu_t);
                     tot = __fadd_rn(tot, mu_t);
                     mu_inc = __fadd_rn(mu_inc, from);
                     // what the winner will need: the new partial sum and the two terms between the
@@ -533,7 +536,8 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 }
                 tot = __fadd_rn(tot, mu_inc);
                 mean = div_small(tot, c + 1);                                // c + 1 <= 9 in this kernel
-                key_hi = decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
+                key_hi = kPlain ? (mean < g.lambda ? __float_as_uint(mean) : 0xffffffffu)
+                                : decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
             }
             // warp argmin: lowest key, then the lowest lane (= lowest GPU index of this warp) that holds it
             const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
@@ -642,7 +646,7 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
         a.matrix_mode = 1; a.pair_cache = 1;
         a.gpus_per_warp = 32;
         const uint32_t threads = 2 * 32 * ((a.G + 31) / 32);                 // owner warps + as many fetch warps
-        auto kern = place_fast_kernel;
+        auto kern = (a.admit_rule == 0 && a.objective == 0) ? place_fast_kernel<true> : place_fast_kernel<false>;
         if (fast_bytes > 48 * 1024)
             ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast_bytes));
         kern<<<num_streams, threads, fast_bytes, st>>>(a);
