@@ -205,7 +205,7 @@ struct TileArgs {
     const uint32_t* tile_counter;
     uint32_t tile_capacity;
     TilePartial* partials;
-    const float* inv_table;      // [2W + 1] 1/s
+    const float* inv_table;      // [2W + 1] 1/s (LOCKSTEP tiles only)
     uint32_t n_inv;              // 2W + 1
     PhiCap cap;
     uint32_t* status;            // library status word (sticky flags)
@@ -311,7 +311,8 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
 
-// copies of one tile: chunk c of A goes to slots 17c.., chunk c of B to slots 17 (b_off/16 + c)..
+// copies of one tile: chunk c of A goes to the slots from (kChunk + 1) c on, chunk c of B to those from
+// (kChunk + 1) (b_off / kChunk + c) on
 __device__ __forceinline__ void stage_tile_async(const uint4* __restrict__ records, const TileDesc& d, uint32_t loadA,
                                                  uint32_t loadB, uint32_t b_off, uint4* s_rec, uint64_t* bar) {
     const uint32_t nA = (loadA + kChunk - 1) / kChunk, nB = (loadB + kChunk - 1) / kChunk;
