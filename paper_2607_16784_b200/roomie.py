@@ -36,7 +36,7 @@ def lib_path() -> str:
 def _load():
     if not os.path.exists(_LIB_PATH):
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2607_16784_b200.build` "
+            f"{_LIB_PATH} is missing: build it with `python paper_2607_16784_b200/build.py` "
             "(nvcc, sm_100a).  This package has no CPU or PyTorch fallback.")
     dll = C.CDLL(_LIB_PATH)
     dll.roomie_strerror.restype = C.c_char_p

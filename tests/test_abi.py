@@ -13,7 +13,10 @@ def _declared():
 
 
 def test_library_exports_every_declared_symbol():
-    from paper_2607_16784_b200 import build
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("_roomie_build", os.path.join(ROOT, "paper_2607_16784_b200", "build.py"))
+    build = importlib.util.module_from_spec(spec)                  # by path: the package itself needs the library
+    spec.loader.exec_module(build)
     path = build.build()
     dll = ctypes.CDLL(path)
     names = _declared()
