@@ -28,13 +28,23 @@ struct DetailedArgs {
 
 struct BlockNeed { uint32_t wb, regs, smem, b; };
 
+// floor(a / d) for a < 2^23, d >= 1 without the integer-division routine (about 20 instructions, several
+// per simulated event): approximate float quotient, then one exact correction step in integers
+__device__ __forceinline__ uint32_t div_floor(uint32_t a, uint32_t d) {
+    uint32_t q = (uint32_t)__fdividef((float)a, (float)d);            // within 1 of the true quotient
+    const int32_t r = (int32_t)a - (int32_t)(q * d);
+    if (r < 0) --q;
+    else if ((uint32_t)r >= d) ++q;
+    return q;
+}
+
 __device__ __forceinline__ BlockNeed need_of(const uint4& r) {
     BlockNeed n;
     n.b = r.w >> 22;
     const uint32_t warps = r.z >> kWarpShift, regs = r.z & ((1u << kWarpShift) - 1u), smem = r.w & ((1u << 22) - 1u);
-    n.wb = n.b ? warps / n.b : 0u;
-    n.regs = n.b ? regs / n.b : 0u;
-    n.smem = n.b ? smem / n.b : 0u;
+    n.wb = n.b ? div_floor(warps, n.b) : 0u;
+    n.regs = n.b ? div_floor(regs, n.b) : 0u;
+    n.smem = n.b ? div_floor(smem, n.b) : 0u;
     return n;
 }
 
@@ -42,9 +52,9 @@ __device__ __forceinline__ BlockNeed need_of(const uint4& r) {
 __device__ __forceinline__ uint32_t blocks_in(const BlockNeed& n, uint32_t warps, uint32_t regs, uint32_t smem,
                                               uint32_t slots) {
     uint32_t b = n.b;
-    if (n.wb) b = min(b, warps / n.wb);
-    if (n.regs) b = min(b, regs / n.regs);
-    if (n.smem) b = min(b, smem / n.smem);
+    if (n.wb) b = min(b, div_floor(warps, n.wb));
+    if (n.regs) b = min(b, div_floor(regs, n.regs));
+    if (n.smem) b = min(b, div_floor(smem, n.smem));
     return min(b, slots);
 }
 
