@@ -28,6 +28,23 @@ struct DetailedArgs {
 
 struct BlockNeed { uint32_t wb, regs, smem, b; };
 
+// b~ / b for b~ <= b <= kRateMax, correctly rounded by the host compiler: the progress rate of a kernel that
+// keeps b~ of its b blocks.  One load instead of the double-precision division routine; larger b (more than
+// 32 resident blocks per SM) take the division.
+constexpr int kRateMax = 32;
+struct RateTable {
+    double v[(kRateMax + 1) * (kRateMax + 1)];
+    constexpr RateTable() : v{} {
+        for (int i = 0; i <= kRateMax; ++i)
+            for (int j = 1; j <= kRateMax; ++j) v[i * (kRateMax + 1) + j] = (double)i / (double)j;
+    }
+};
+__device__ const RateTable kRates = RateTable();
+__device__ __forceinline__ double rate_of(uint32_t kept, uint32_t all) {
+    if (all <= (uint32_t)kRateMax) return __ldg(&kRates.v[kept * (kRateMax + 1) + all]);
+    return __ddiv_rn((double)kept, (double)all);
+}
+
 // floor(a / d) for a < 2^23, d >= 1 without the integer-division routine (about 20 instructions, several
 // per simulated event): approximate float quotient, then one exact correction step in integers
 __device__ __forceinline__ uint32_t div_floor(uint32_t a, uint32_t d) {
@@ -106,8 +123,8 @@ __global__ void __launch_bounds__(128) detailed_walk_kernel(DetailedArgs g) {
                         b0 = first0 ? n0.b : bl;
                         b1 = first0 ? bl : n1.b;
                     }
-                    rate[0] = __ddiv_rn((double)b0, (double)n0.b);
-                    rate[1] = __ddiv_rn((double)b1, (double)n1.b);
+                    rate[0] = rate_of(b0, n0.b);
+                    rate[1] = rate_of(b1, n1.b);
                 }
                 double t[2];
 #pragma unroll
