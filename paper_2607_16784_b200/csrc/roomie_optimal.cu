@@ -22,7 +22,16 @@ struct OptArgs {
     uint32_t n, S, G, R;
     unsigned long long* best_key;   // [S] (cost bits << 32) | code, smaller is better
     unsigned long long n_prefix;    // G^(n-2) (1 when n <= 2)
+    double inv_n;                   // the double nearest to 1/n
 };
+
+// c / n, correctly rounded like the float32 division it stands for, for n <= 16: the double product of c and
+// the double nearest to 1/n is within 2^-52 (relative) of c/n, while the quotient of a 24-bit c by such an n
+// is either a float or at least 2^-30 (relative) away from the midpoint of two neighbouring floats, so
+// rounding the product to float32 rounds the quotient.  Larger n take the division.
+__device__ __forceinline__ float div_by_n(float c, double inv_n, float fn) {
+    return fn <= 16.0f ? __double2float_rn(__dmul_rn((double)c, inv_n)) : __fdiv_rn(c, fn);
+}
 
 // pair sums s[i][j] = P[m_i][m_j] + P[m_j][m_i] of one scenario into shared memory
 __device__ __forceinline__ void load_pair_sums(const OptArgs& g, const int32_t* models, float* s_pair) {
@@ -42,17 +51,28 @@ __global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs
     __syncthreads();
     unsigned long long best = ~0ull;
     const float fn = (float)n;
+    const double inv_n = g.inv_n;
     for (unsigned long long pc = (unsigned long long)blockIdx.x * kOptThreads + threadIdx.x; pc < g.n_prefix;
          pc += (unsigned long long)gridDim.x * kOptThreads) {
         // digits of the prefix code: model 1 is the most significant one; 4 bits per model / per GPU load
         unsigned long long assign = 0, load = 1;                    // model 0 on GPU 0
-        unsigned long long rest = pc;
         bool ok = true;
-        for (int k = (int)n - 2; k >= 1; --k) {
-            const uint32_t d = (uint32_t)(rest % G);
-            rest /= G;
-            assign |= (unsigned long long)d << (4 * k);
-            load += 1ull << (4 * d);
+        if (pc >> 32) {                                             // 64-bit division only for codes that need it
+            unsigned long long rest = pc;
+            for (int k = (int)n - 2; k >= 1; --k) {
+                const uint32_t d = (uint32_t)(rest % G);
+                rest /= G;
+                assign |= (unsigned long long)d << (4 * k);
+                load += 1ull << (4 * d);
+            }
+        } else {
+            uint32_t rest = (uint32_t)pc;
+            for (int k = (int)n - 2; k >= 1; --k) {
+                const uint32_t q = rest / G, d = rest - q * G;
+                rest = q;
+                assign |= (unsigned long long)d << (4 * k);
+                load += 1ull << (4 * d);
+            }
         }
         for (uint32_t d = 0; d < G; ++d) ok = ok && ((load >> (4 * d)) & 15ull) <= R;
         if (!ok) continue;
@@ -72,7 +92,7 @@ __global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs
             for (uint32_t i = 0; i + 1 < n; ++i)
                 if (((uint32_t)(assign >> (4 * i)) & 15u) == d) c = __fadd_rn(c, s_pair[i * n + (n - 1)]);
             const unsigned long long code = pc * G + d;
-            const unsigned long long key = ((unsigned long long)__float_as_uint(__fdiv_rn(c, fn)) << 32) | code;
+            const unsigned long long key = ((unsigned long long)__float_as_uint(div_by_n(c, inv_n, fn)) << 32) | code;
             best = key < best ? key : best;
         }
     }
@@ -150,7 +170,7 @@ extern "C" int roomie_optimal_assignment(const float* Pmat, uint32_t P, const in
     ROOMIE_CUDA_OK(cudaMemsetAsync(keys, 0xFF, 8 * (size_t)num_scenarios, st));
     OptArgs a;
     a.Pm = Pmat; a.P = P; a.models = models; a.n = n; a.S = num_scenarios; a.G = num_gpus; a.R = max_residents;
-    a.best_key = keys; a.n_prefix = prefix;
+    a.best_key = keys; a.n_prefix = prefix; a.inv_n = 1.0 / (double)n;
     unsigned long long ctas = (prefix + kOptThreads - 1) / kOptThreads;
     const unsigned long long cap = (unsigned long long)sm_count() * 8;      // enough CTAs to fill the GPU per scenario
     if (ctas > cap) ctas = cap;
