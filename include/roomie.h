@@ -327,6 +327,14 @@ const char *roomie_last_cuda_error(void);
 uint64_t roomie_launch_count(void);
 void roomie_reset_launch_count(void);
 
+/* Self-test of the library's bounded waits (the paper has no counterpart).  The pairwise walk stages its
+ * tiles with asynchronous copies and waits for them on a barrier, with a time limit; a wait that runs out
+ * sets ROOMIE_FLAG_WAIT_TIMEOUT in the library's status word and ends the CTA instead of hanging the GPU.
+ * This call launches one CTA that waits, with `limit_ns` (1 .. 1e9) as the limit, for a copy that is never
+ * issued: afterwards *status (device word, e.g. roomie_library.status or a word of the caller's) has
+ * ROOMIE_FLAG_WAIT_TIMEOUT set and the context is still usable.  Errors: INVALID_ARG, CUDA. */
+int roomie_selftest_bounded_wait(uint32_t *status /* device */, uint64_t limit_ns, void *stream);
+
 /* Measurement aid (the paper has no counterpart).  While enabled, the calling thread's pair
  * calls bracket every launch of the pairwise walk kernel with a pair of CUDA events recorded on
  * the call's stream (at most 256 pairs are kept; later launches are not recorded).

@@ -11,6 +11,7 @@ There is no CPU fallback: importing this package without the compiled library ra
 from .roomie import (  # noqa: F401
     GpuSpec, Library, ClusterState, RoomieError, TIMELINE, LOCKSTEP, DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS,
     occupancy, library_build, pair_workspace_bytes, pair_matrix, pair_interference, pair_interference_static,
-    multi_estimate, place, place_batch, optimal_assignment, assignment_cost, launch_count, reset_launch_count, profile_enable, profile_walk_ms, lib_path, EXPORTS,
+    multi_estimate, place, place_batch, optimal_assignment, assignment_cost, launch_count, reset_launch_count, profile_enable, profile_walk_ms,
+    selftest_bounded_wait, lib_path, EXPORTS,
 )
 from .shard import partition_pairs, combine_shards, pair_matrix_sharded  # noqa: F401,E402

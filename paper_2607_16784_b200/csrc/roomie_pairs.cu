@@ -296,12 +296,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // waits for the phase with the given parity; gives up after kWaitNs (and, should the timer not
 // advance, after kWaitSpins polls)
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, unsigned long long limit_ns = kWaitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > kWaitNs) return false;
+        if (global_ns() - t0 > limit_ns) return false;
     }
     return false;
 }
@@ -429,6 +429,20 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
     }
 }
 #undef ROOMIE_WALK_STEP
+
+// Self-test of the bounded wait: one CTA announces 16 bytes on a barrier, issues no copy, and waits
+// with the given limit.  The wait must run out; the kernel then raises the same status bit a real
+// time-out raises and returns, leaving the context usable.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(uint32_t* status, unsigned long long limit_ns) {
+    __shared__ __align__(8) uint64_t s_bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&s_bar, 1);
+        mbar_arrive_expect(&s_bar, 16);
+    }
+    __syncwarp();
+    const bool arrived = mbar_wait_bounded(&s_bar, 0, limit_ns);
+    if (!__all_sync(0xffffffffu, arrived) && threadIdx.x == 0) atomicOr(status, ROOMIE_FLAG_WAIT_TIMEOUT);
+}
 
 // ---------------------------------------------------------------------------------------
 // LOCKSTEP tiles (Algorithm 1 as printed): pairing t of the walk is (s_i + t, s_j + t)
@@ -857,6 +871,14 @@ static int static_scratch_for_current_device(void** out) {
     return ROOMIE_OK;
 }
 }  // namespace roomie
+
+extern "C" int roomie_selftest_bounded_wait(uint32_t* status, uint64_t limit_ns, void* stream) {
+    if (!status || limit_ns == 0 || limit_ns > 1000000000ull) return ROOMIE_ERR_INVALID_ARG;
+    wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status, limit_ns);
+    note_launch();
+    ROOMIE_CUDA_OK(cudaGetLastError());
+    return ROOMIE_OK;
+}
 
 extern "C" size_t roomie_pair_workspace_bytes(const roomie_library* lib, const roomie_opts* opts,
                                               uint64_t pair_begin, uint64_t pair_end) {

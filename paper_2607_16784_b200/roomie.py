@@ -17,7 +17,7 @@ DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS = 2, 3, 4
 EXPORTS = [
     "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
-    "roomie_pair_interference_workspace_bytes",
+    "roomie_pair_interference_workspace_bytes", "roomie_selftest_bounded_wait",
     "roomie_pair_interference_static",
     "roomie_multi_estimate", "roomie_place", "roomie_place_batch", "roomie_optimal_workspace_bytes",
     "roomie_optimal_assignment", "roomie_assignment_cost", "roomie_strerror", "roomie_last_cuda_error",
@@ -45,6 +45,7 @@ def _load():
     dll.roomie_share_table_floats.restype = C.c_size_t
     dll.roomie_pair_workspace_bytes.restype = C.c_size_t
     dll.roomie_pair_workspace_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64]
+    dll.roomie_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
     dll.roomie_pair_interference_workspace_bytes.restype = C.c_size_t
     dll.roomie_pair_interference_workspace_bytes.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p]
     dll.roomie_pair_matrix.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p,
@@ -423,6 +424,15 @@ def launch_count() -> int:
 
 def reset_launch_count():
     _dll.roomie_reset_launch_count()
+
+
+def selftest_bounded_wait(limit_ns: int = 1_000_000, stream=None) -> int:
+    """roomie_selftest_bounded_wait: one CTA waits `limit_ns` for a copy nobody issues.  Returns the status
+    word afterwards (ROOMIE_FLAG_WAIT_TIMEOUT = 8 must be set)."""
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(_dll.roomie_selftest_bounded_wait(_ptr(word), C.c_uint64(int(limit_ns)), _stream(stream)),
+           "roomie_selftest_bounded_wait")
+    return int(word.item())
 
 
 def profile_enable(on: bool = True):

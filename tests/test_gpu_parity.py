@@ -623,3 +623,24 @@ def test_timelines_close_to_the_tick_limit(rm, oracle):
         assert_close(got.cpu().numpy(), want)
     for a, b in ((0, 1), (2, 1)):
         check_pair_detail(rm, oracle, ol, gl, a, b, mode=0, n_align=8, start_filter=0)
+
+
+def test_bounded_wait_gives_up_and_leaves_the_context_usable(rm, oracle):
+    """The walk kernel waits for its tile copies on a barrier with a time limit.  The self-test waits 2 ms for a
+    copy that is never issued: the wait must run out, raise the status bit a real time-out raises, and the next
+    calls must work as if nothing had happened."""
+    import time
+    import torch
+    t0 = time.perf_counter()
+    flags = rm.selftest_bounded_wait(2_000_000)
+    torch.cuda.synchronize()
+    assert flags == 8                                   # ROOMIE_FLAG_WAIT_TIMEOUT and nothing else
+    assert time.perf_counter() - t0 < 5.0
+    with pytest.raises(rm.RoomieError):
+        rm.selftest_bounded_wait(0)
+    lib = rs.make_library(0)
+    ol, gl = build_both(rm, oracle, lib)
+    want, wev = oracle.pair_matrix(ol, mode=0, n_align=8, start_filter=1)
+    got, ev = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)
+    assert gl.status_flags() == 0 and int(ev.item()) == wev
+    assert_close(got.cpu().numpy(), want)
