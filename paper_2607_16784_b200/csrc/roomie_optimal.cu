@@ -6,8 +6,8 @@
 //     cost = ( sum over i < j on the same GPU of (P[m_i][m_j] + P[m_j][m_i]) ) / n,
 // defined in float32: pair terms are accumulated model by model (j ascending, partners i < j
 // ascending), one division at the end.  That order lets the search share work: a thread fixes the
-// GPUs of models 1..n-2 (model 0 sits on GPU 0), sums their terms once, and only adds the last
-// model's terms for each of its G choices.
+// GPUs of models 1..n-3 (model 0 sits on GPU 0), sums their terms once, adds the terms of model n-2
+// once for each of its G choices and those of the last model for each of the G*G choices of both.
 #include "roomie_common.cuh"
 
 namespace roomie {
@@ -21,7 +21,7 @@ struct OptArgs {
     const int32_t* models;          // [S][n]
     uint32_t n, S, G, R;
     unsigned long long* best_key;   // [S] (cost bits << 32) | code, smaller is better
-    unsigned long long n_prefix;    // G^(n-2) (1 when n <= 2)
+    unsigned long long n_prefix;    // G^(n-3): codes of the models a thread does not enumerate itself (1 when n <= 3)
     double inv_n;                   // the double nearest to 1/n
 };
 
@@ -52,14 +52,18 @@ __global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs
     unsigned long long best = ~0ull;
     const float fn = (float)n;
     const double inv_n = g.inv_n;
+    // A thread fixes the GPUs of models 1 .. n-1-kTail (prefix code pc, model 1 the most significant digit) and
+    // tries every choice of the last kTail models below it: kTail = 2 when there are at least three models, so
+    // that the prefix's digits, feasibility and pair terms are paid once per G*G assignments, not once per G.
+    const uint32_t tail = n >= 3 ? 2u : n - 1u;                     // n = 2: one tail model; n = 1: none
+    const uint32_t n_fix = n - tail;                                 // models 0 .. n_fix-1 are fixed by the prefix
     for (unsigned long long pc = (unsigned long long)blockIdx.x * kOptThreads + threadIdx.x; pc < g.n_prefix;
          pc += (unsigned long long)gridDim.x * kOptThreads) {
-        // digits of the prefix code: model 1 is the most significant one; 4 bits per model / per GPU load
+        // digits of the prefix code; 4 bits per model (its GPU) and per GPU (its load)
         unsigned long long assign = 0, load = 1;                    // model 0 on GPU 0
-        bool ok = true;
         if (pc >> 32) {                                             // 64-bit division only for codes that need it
             unsigned long long rest = pc;
-            for (int k = (int)n - 2; k >= 1; --k) {
+            for (int k = (int)n_fix - 1; k >= 1; --k) {
                 const uint32_t d = (uint32_t)(rest % G);
                 rest /= G;
                 assign |= (unsigned long long)d << (4 * k);
@@ -67,33 +71,48 @@ __global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs
             }
         } else {
             uint32_t rest = (uint32_t)pc;
-            for (int k = (int)n - 2; k >= 1; --k) {
+            for (int k = (int)n_fix - 1; k >= 1; --k) {
                 const uint32_t q = rest / G, d = rest - q * G;
                 rest = q;
                 assign |= (unsigned long long)d << (4 * k);
                 load += 1ull << (4 * d);
             }
         }
+        bool ok = true;
         for (uint32_t d = 0; d < G; ++d) ok = ok && ((load >> (4 * d)) & 15ull) <= R;
         if (!ok) continue;
-        float tot = 0.0f;                                           // terms among models 0 .. n-2
-        for (uint32_t j = 1; j + 1 < n; ++j) {
+        float tot = 0.0f;                                           // terms among the fixed models
+        for (uint32_t j = 1; j < n_fix; ++j) {
             const uint32_t gj = (uint32_t)(assign >> (4 * j)) & 15u;
             for (uint32_t i = 0; i < j; ++i)
                 if (((uint32_t)(assign >> (4 * i)) & 15u) == gj) tot = __fadd_rn(tot, s_pair[i * n + j]);
         }
-        if (n == 1) {
+        if (tail == 0) {
             best = 0ull;                                            // a single model: cost 0, code 0
             continue;
         }
-        for (uint32_t d = 0; d < G; ++d) {                          // the last model's GPU
-            if (((load >> (4 * d)) & 15ull) >= R) continue;
-            float c = tot;
-            for (uint32_t i = 0; i + 1 < n; ++i)
-                if (((uint32_t)(assign >> (4 * i)) & 15u) == d) c = __fadd_rn(c, s_pair[i * n + (n - 1)]);
-            const unsigned long long code = pc * G + d;
-            const unsigned long long key = ((unsigned long long)__float_as_uint(div_by_n(c, inv_n, fn)) << 32) | code;
-            best = key < best ? key : best;
+        // tail model a = n_fix (only when tail == 2), then the last model n-1
+        const uint32_t g2_count = tail == 2 ? G : 1u;
+        for (uint32_t d2 = 0; d2 < g2_count; ++d2) {
+            unsigned long long assign2 = assign, load2 = load, code2 = pc;
+            float tot2 = tot;
+            if (tail == 2) {
+                if (((load >> (4 * d2)) & 15ull) >= R) continue;
+                for (uint32_t i = 0; i < n_fix; ++i)
+                    if (((uint32_t)(assign >> (4 * i)) & 15u) == d2) tot2 = __fadd_rn(tot2, s_pair[i * n + n_fix]);
+                assign2 |= (unsigned long long)d2 << (4 * n_fix);
+                load2 += 1ull << (4 * d2);
+                code2 = pc * G + d2;
+            }
+            for (uint32_t d = 0; d < G; ++d) {                      // the last model's GPU
+                if (((load2 >> (4 * d)) & 15ull) >= R) continue;
+                float c = tot2;
+                for (uint32_t i = 0; i + 1 < n; ++i)
+                    if (((uint32_t)(assign2 >> (4 * i)) & 15u) == d) c = __fadd_rn(c, s_pair[i * n + (n - 1)]);
+                const unsigned long long code = code2 * G + d;
+                const unsigned long long key = ((unsigned long long)__float_as_uint(div_by_n(c, inv_n, fn)) << 32) | code;
+                best = key < best ? key : best;
+            }
         }
     }
 #pragma unroll
@@ -160,9 +179,10 @@ extern "C" int roomie_optimal_assignment(const float* Pmat, uint32_t P, const in
     if (workspace_bytes < roomie_optimal_workspace_bytes(num_scenarios)) return ROOMIE_ERR_CAPACITY;
     // the code of an assignment (base-G digits of models 1..n-1) must fit 32 bits
     unsigned long long codes = 1, prefix = 1;
+    const uint32_t tail = n >= 3 ? 2u : n - 1u;                     // models enumerated inside a thread
     for (uint32_t k = 1; k < n; ++k) {
         codes *= num_gpus;
-        if (k + 1 < n) prefix *= num_gpus;
+        if (k + tail < n) prefix *= num_gpus;
         if (codes > (1ull << 32)) return ROOMIE_ERR_CAPACITY;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);

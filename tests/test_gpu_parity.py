@@ -474,7 +474,7 @@ def test_optimal_assignment_bit_exact(rm, oracle):
     _, gl = build_both(rm, oracle, lib)
     Pm32 = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)[0].cpu().numpy()
     P = Pm32.shape[0]
-    for n, G, R, S in ((1, 3, 2, 3), (2, 1, 2, 3), (5, 2, 3, 20), (7, 3, 3, 12), (8, 4, 2, 6), (9, 3, 3, 4), (4, 2, 1, 2)):
+    for n, G, R, S in ((1, 3, 2, 3), (2, 1, 2, 3), (2, 3, 1, 3), (3, 2, 2, 4), (3, 3, 1, 3), (5, 2, 3, 20), (7, 3, 3, 12), (8, 4, 2, 6), (9, 3, 3, 4), (4, 2, 1, 2)):
         models = rng.integers(0, P, (S, n)).astype(np.int32)
         cost, assign = rm.optimal_assignment(Pm32, models, G, R)
         cost, assign = cost.cpu().numpy(), assign.cpu().numpy()
