@@ -6,14 +6,16 @@
 //     cost = ( sum over i < j on the same GPU of (P[m_i][m_j] + P[m_j][m_i]) ) / n,
 // defined in float32: pair terms are accumulated model by model (j ascending, partners i < j
 // ascending), one division at the end.  That order lets the search share work: a thread fixes the
-// GPUs of models 1..n-3 (model 0 sits on GPU 0), sums their terms once, adds the terms of model n-2
-// once for each of its G choices and those of the last model for each of the G*G choices of both.
+// GPUs of models 1..n-3 (model 0 sits on GPU 0), sums their terms once, and enumerates the last two
+// models itself; for each of them one pass over the earlier models yields the sums of all G choices
+// (a running sum per GPU, every one taking its members' terms in ascending order).
 #include "roomie_common.cuh"
 
 namespace roomie {
 
 constexpr int kOptThreads = 256;
 constexpr int kOptMaxModels = 16;
+constexpr int kOptMaxGpus = 15;
 
 struct OptArgs {
     const float* Pm;
@@ -46,6 +48,9 @@ __device__ __forceinline__ void load_pair_sums(const OptArgs& g, const int32_t* 
 __global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs g) {
     __shared__ float s_pair[kOptMaxModels * kOptMaxModels];
     __shared__ unsigned long long s_best[kOptThreads / 32];
+    __shared__ float s_acc[2][kOptMaxGpus * kOptThreads];           // per-GPU running sums of the two tail models
+    float* acc1 = s_acc[0] + threadIdx.x;
+    float* acc2 = s_acc[1] + threadIdx.x;
     const uint32_t sc = blockIdx.y, n = g.n, G = g.G, R = g.R;
     load_pair_sums(g, g.models + (size_t)sc * n, s_pair);
     __syncthreads();
@@ -91,26 +96,38 @@ __global__ void __launch_bounds__(kOptThreads) optimal_assignment_kernel(OptArgs
             best = 0ull;                                            // a single model: cost 0, code 0
             continue;
         }
-        // tail model a = n_fix (only when tail == 2), then the last model n-1
+        // One pass over the models gives the sums for all G choices of a tail model at once: every GPU's
+        // accumulator starts from the sum so far and takes the terms of its own members in ascending
+        // order, which is exactly the order of the definition.  The accumulators live in shared memory
+        // ([gpu][thread], so the threads of a warp touch consecutive words).
+        if (tail == 2) {                                            // model n_fix
+            for (uint32_t d = 0; d < G; ++d) acc2[d * kOptThreads] = tot;
+            for (uint32_t i = 0; i < n_fix; ++i) {
+                float* a2 = acc2 + ((uint32_t)(assign >> (4 * i)) & 15u) * kOptThreads;
+                *a2 = __fadd_rn(*a2, s_pair[i * n + n_fix]);
+            }
+        }
         const uint32_t g2_count = tail == 2 ? G : 1u;
         for (uint32_t d2 = 0; d2 < g2_count; ++d2) {
             unsigned long long assign2 = assign, load2 = load, code2 = pc;
             float tot2 = tot;
             if (tail == 2) {
                 if (((load >> (4 * d2)) & 15ull) >= R) continue;
-                for (uint32_t i = 0; i < n_fix; ++i)
-                    if (((uint32_t)(assign >> (4 * i)) & 15u) == d2) tot2 = __fadd_rn(tot2, s_pair[i * n + n_fix]);
+                tot2 = acc2[d2 * kOptThreads];
                 assign2 |= (unsigned long long)d2 << (4 * n_fix);
                 load2 += 1ull << (4 * d2);
                 code2 = pc * G + d2;
             }
-            for (uint32_t d = 0; d < G; ++d) {                      // the last model's GPU
+            for (uint32_t d = 0; d < G; ++d) acc1[d * kOptThreads] = tot2;      // the last model
+            for (uint32_t i = 0; i + 1 < n; ++i) {
+                float* a1 = acc1 + ((uint32_t)(assign2 >> (4 * i)) & 15u) * kOptThreads;
+                *a1 = __fadd_rn(*a1, s_pair[i * n + (n - 1)]);
+            }
+            for (uint32_t d = 0; d < G; ++d) {
                 if (((load2 >> (4 * d)) & 15ull) >= R) continue;
-                float c = tot2;
-                for (uint32_t i = 0; i + 1 < n; ++i)
-                    if (((uint32_t)(assign2 >> (4 * i)) & 15u) == d) c = __fadd_rn(c, s_pair[i * n + (n - 1)]);
                 const unsigned long long code = code2 * G + d;
-                const unsigned long long key = ((unsigned long long)__float_as_uint(div_by_n(c, inv_n, fn)) << 32) | code;
+                const unsigned long long key =
+                    ((unsigned long long)__float_as_uint(div_by_n(acc1[d * kOptThreads], inv_n, fn)) << 32) | code;
                 best = key < best ? key : best;
             }
         }
@@ -173,7 +190,7 @@ extern "C" int roomie_optimal_assignment(const float* Pmat, uint32_t P, const in
                                          float* best_cost, int32_t* best_assign, void* workspace,
                                          size_t workspace_bytes, void* stream) {
     if (!Pmat || P == 0 || !models || !best_cost || !workspace || n == 0 || n > kOptMaxModels || num_gpus == 0 ||
-        num_gpus > 15 || max_residents == 0 || max_residents > 15)
+        num_gpus > (uint32_t)kOptMaxGpus || max_residents == 0 || max_residents > 15)
         return ROOMIE_ERR_INVALID_ARG;
     if (num_scenarios == 0) return ROOMIE_OK;
     if (workspace_bytes < roomie_optimal_workspace_bytes(num_scenarios)) return ROOMIE_ERR_CAPACITY;
