@@ -89,6 +89,14 @@ int roomie_occupancy(const roomie_kernel_table *table /* host struct of device a
                      const roomie_gpu_spec *spec /* host */, const roomie_occ_out *out /* host struct */,
                      void *stream);
 
+/* Which kernel roomie_occupancy launches for these arguments (host arithmetic on the pointer values and
+ * n only; nothing is dereferenced, no CUDA call is made; the paper has no counterpart).  Arrays need only
+ * their elements' own 4-byte alignment: bit 0 of the result is set when the 128-bit kernel is used, which
+ * takes n >= 4 and every input column and every packed4 / occ / occ_theo output (NULL counts as aligned) on
+ * a 16-byte boundary; bits 4-7 tell which of the four rows of phi (row c starts at phi + c*n) take 128-bit
+ * stores there.  0 = the scalar kernel.  Negative: ROOMIE_ERR_INVALID_ARG (NULL struct). */
+int roomie_occupancy_variant(const roomie_kernel_table *table /* host */, const roomie_occ_out *out /* host */);
+
 /* A kernel library prepared for the interference walk.  The caller allocates every array and
  * fills the struct (host memory); roomie_library_build writes the device arrays.
  * Record layout (16 bytes per kernel, the unit the walk streams):

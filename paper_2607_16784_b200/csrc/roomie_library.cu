@@ -29,11 +29,12 @@ __device__ __forceinline__ void occ_store_scalar(const OccArgs& a, uint32_t k, c
     }
 }
 
-// kVec: inputs and the packed / occ / occ_theo outputs are 16-byte aligned, so the first n/4*4 kernels go
-// four per thread with 128-bit accesses (the up to three left over are done one by one);
-// kVecPhi: n is a multiple of 4 as well, so the four component arrays of phi are aligned too.
-template <bool kVec, bool kVecPhi>
-__global__ void __launch_bounds__(256) occupancy_kernel(OccArgs a) {
+// kVec: the four input columns and the packed / occ / occ_theo outputs are 16-byte aligned, so the first
+// n/4*4 kernels go four per thread with 128-bit accesses (the up to three left over are done one by one).
+// Row c of phi starts at phi + c*n, so whether it can take 128-bit stores depends on n as well as on the
+// pointer: `phi_rows` has bit c set when that row is 16-byte aligned; the other rows get four scalar stores.
+template <bool kVec>
+__global__ void __launch_bounds__(256) occupancy_kernel(OccArgs a, uint32_t phi_rows) {
     uint32_t bad = 0;
     const uint32_t n4 = kVec ? a.n / 4 : 0;
     if (kVec) {
@@ -63,21 +64,15 @@ __global__ void __launch_bounds__(256) occupancy_kernel(OccArgs a) {
                 reinterpret_cast<float4*>(a.occ_theo)[i] =
                     make_float4(o[0].occ_theo, o[1].occ_theo, o[2].occ_theo, o[3].occ_theo);
             if (a.phi) {
-                if (kVecPhi) {
-                    uint4* p = reinterpret_cast<uint4*>(a.phi);
-                    p[i] = make_uint4(o[0].warps, o[1].warps, o[2].warps, o[3].warps);
-                    p[n4 + i] = make_uint4(o[0].phi_regs, o[1].phi_regs, o[2].phi_regs, o[3].phi_regs);
-                    p[2 * (size_t)n4 + i] = make_uint4(o[0].phi_smem, o[1].phi_smem, o[2].phi_smem, o[3].phi_smem);
-                    p[3 * (size_t)n4 + i] = make_uint4(o[0].b_res, o[1].b_res, o[2].b_res, o[3].b_res);
-                } else {
+                const uint4 rows[4] = {make_uint4(o[0].warps, o[1].warps, o[2].warps, o[3].warps),
+                                       make_uint4(o[0].phi_regs, o[1].phi_regs, o[2].phi_regs, o[3].phi_regs),
+                                       make_uint4(o[0].phi_smem, o[1].phi_smem, o[2].phi_smem, o[3].phi_smem),
+                                       make_uint4(o[0].b_res, o[1].b_res, o[2].b_res, o[3].b_res)};
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const size_t k = 4 * (size_t)i + j;
-                        a.phi[k] = o[j].warps;
-                        a.phi[(size_t)a.n + k] = o[j].phi_regs;
-                        a.phi[2 * (size_t)a.n + k] = o[j].phi_smem;
-                        a.phi[3 * (size_t)a.n + k] = o[j].b_res;
-                    }
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t* row = a.phi + (size_t)c * a.n + 4 * (size_t)i;
+                    if (phi_rows & (1u << c)) *reinterpret_cast<uint4*>(row) = rows[c];
+                    else { row[0] = rows[c].x; row[1] = rows[c].y; row[2] = rows[c].z; row[3] = rows[c].w; }
                 }
             }
         }
@@ -192,6 +187,22 @@ __global__ void share_table_kernel(float* tab, uint32_t n) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Which occupancy kernel a call gets (pointers are only looked at, never dereferenced):
+//   bit 0     the 128-bit kernel: n >= 4 and every input column and every packed / occ / occ_theo output
+//             (a NULL output counts as aligned) sits on a 16-byte boundary; otherwise the scalar kernel,
+//             which has no alignment requirement beyond the element's own;
+//   bits 4-7  rows of phi ([4][n]) that take 128-bit stores inside that kernel: row c starts at phi + c*n.
+static int occupancy_variant_of(const roomie_kernel_table* t, const roomie_occ_out* o) {
+    const bool vec = t->n >= 4 && aligned16(t->grid_blocks) && aligned16(t->block_threads) &&
+                     aligned16(t->regs_per_thread) && aligned16(t->smem_per_block) && aligned16(o->packed4) &&
+                     aligned16(o->occ) && aligned16(o->occ_theo);
+    if (!vec) return 0;
+    int rows = 0;
+    for (int c = 0; c < 4; ++c)
+        if (o->phi && aligned16(o->phi + (size_t)c * t->n)) rows |= 1 << c;
+    return 1 | (rows << 4);
+}
+
 int validate_spec(const roomie_gpu_spec* s) {
     if (!s) return ROOMIE_ERR_INVALID_ARG;
     if (s->num_sms == 0 || s->threads_per_sm < 32) return ROOMIE_ERR_INVALID_ARG;
@@ -219,21 +230,22 @@ extern "C" int roomie_occupancy(const roomie_kernel_table* table, const roomie_g
     a.packed4 = out->packed4; a.occ = out->occ; a.occ_theo = out->occ_theo; a.phi = out->phi;
     a.n_unlaunchable = out->n_unlaunchable;
     a.n = table->n; a.spec = *spec;
-    // the 128-bit variant pays off only when phi can be stored with 128-bit accesses too (n a multiple of 4 or no
-    // phi output): four scalar stores per component at a 16-byte stride waste more than the wide loads gain
-    const bool vec_phi = (a.n % 4 == 0 || !a.phi) && aligned16(a.phi);
-    const bool vec = a.n >= 4 && vec_phi && aligned16(a.grid) && aligned16(a.threads) && aligned16(a.regs) &&
-                     aligned16(a.smem) && aligned16(a.packed4) && aligned16(a.occ) && aligned16(a.occ_theo);
+    const int variant = occupancy_variant_of(table, out);
+    const bool vec = (variant & 1) != 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const uint32_t work = vec ? a.n / 4 : a.n;
+    const uint32_t work = vec ? a.n / 4 + 3 : a.n;
     uint32_t blocks = (work + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    if (vec_phi) occupancy_kernel<true, true><<<blocks, 256, 0, st>>>(a);
-    else if (vec) occupancy_kernel<true, false><<<blocks, 256, 0, st>>>(a);
-    else occupancy_kernel<false, false><<<blocks, 256, 0, st>>>(a);
+    if (vec) occupancy_kernel<true><<<blocks, 256, 0, st>>>(a, (uint32_t)variant >> 4);
+    else occupancy_kernel<false><<<blocks, 256, 0, st>>>(a, 0u);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;
+}
+
+extern "C" int roomie_occupancy_variant(const roomie_kernel_table* table, const roomie_occ_out* out) {
+    if (!table || !out) return ROOMIE_ERR_INVALID_ARG;
+    return occupancy_variant_of(table, out);
 }
 
 extern "C" size_t roomie_share_table_floats(const roomie_gpu_spec* spec) {

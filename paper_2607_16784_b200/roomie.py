@@ -15,7 +15,7 @@ TIMELINE, LOCKSTEP = 0, 1
 DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS = 2, 3, 4
 
 EXPORTS = [
-    "roomie_occupancy", "roomie_share_table_floats", "roomie_library_build",
+    "roomie_occupancy", "roomie_occupancy_variant", "roomie_share_table_floats", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
     "roomie_pair_interference_workspace_bytes", "roomie_selftest_bounded_wait",
     "roomie_pair_interference_static",

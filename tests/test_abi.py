@@ -87,3 +87,36 @@ def test_workspace_size_queries_are_host_only():
                                        ctypes.c_void_p]
     assert dll.roomie_pair_matrix(ctypes.byref(bad), ctypes.byref(opts(0, 1)), 0, 6, fake, None, fake * 16, 1 << 20,
                                   None) == -1                # INVALID_ARG before any CUDA call
+
+
+def test_occupancy_kernel_choice_never_vectorises_a_misaligned_array():
+    """The 128-bit occupancy kernel may only be chosen when every array it touches with 128-bit accesses is
+    16-byte aligned; a table or output that is only 4-byte aligned (one profile's slice of a concatenated table)
+    must get the scalar kernel even when n is a multiple of four.  Pointer values only: nothing is dereferenced."""
+    import paper_2607_16784_b200 as pkg
+    from paper_2607_16784_b200 import roomie as rm
+    dll = ctypes.CDLL(pkg.lib_path())
+    base = 0x7F0000000000
+
+    def variant(n, cols=(0, 0, 0, 0), packed=0, occ=0, theo=0, phi=0, no_phi=False, no_packed=False):
+        step = 1 << 24
+        t = rm._Table(n, *(base + i * step + off for i, off in enumerate(cols)))
+        o = rm._OccOut(None if no_packed else base + 4 * step + packed, base + 5 * step + occ, base + 6 * step + theo,
+                       None if no_phi else base + 7 * step + phi, None)
+        return dll.roomie_occupancy_variant(ctypes.byref(t), ctypes.byref(o))
+
+    assert variant(1024) == 1 | (0xF << 4)                      # everything aligned, n % 4 == 0: all rows wide
+    assert variant(1025) == 1 | (0x1 << 4)                      # row c starts 4*c*n bytes in: only row 0 stays aligned
+    assert variant(1026) == 1 | (0x5 << 4)                      # n % 4 == 2: rows 0 and 2
+    assert variant(1493273) & 1                                 # the benchmark's kernel count takes the wide loads
+    assert variant(1024, no_phi=True) == 1 and variant(1024, no_packed=True) == 1 | (0xF << 4)
+    assert variant(3) == 0                                      # fewer than four kernels
+    for i in range(4):                                          # any input column off by one element
+        cols = [0, 0, 0, 0]
+        cols[i] = 4
+        assert variant(1024, cols=tuple(cols)) == 0
+    for kw in (dict(packed=4), dict(occ=8), dict(theo=12)):     # any 128-bit output off the boundary
+        assert variant(1024, **kw) == 0
+    assert variant(1024, phi=4) == 1                            # phi alone misaligned: wide loads, scalar phi rows
+    assert variant(1023, phi=4) == 1 | (0x2 << 4)               # 4 + 4*1023 = 4096: row 1 happens to be aligned
+    assert dll.roomie_occupancy_variant(None, None) == -1

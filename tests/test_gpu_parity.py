@@ -64,15 +64,26 @@ def test_occupancy_bit_exact(rm, oracle, cfg):
 def test_occupancy_ragged_and_unaligned(rm, oracle):
     lib = rs.make_library(1, feasible=False)
     import torch
-    for n in (1, 3, 5, 1023, 1025):
-        # offset by one element: not 16-byte aligned -> scalar kernel; n % 4 != 0 -> scalar kernel
-        cols = [torch.from_numpy(np.ascontiguousarray(x[:n + 1]).view(np.int32)).cuda()[1:]
-                for x in (lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block)]
-        got = rm.occupancy(*cols, lib.spec)
-        want = oracle.occupancy(lib.grid_blocks[1:n + 1], lib.block_threads[1:n + 1],
-                                lib.regs_per_thread[1:n + 1], lib.smem_per_block[1:n + 1], lib.spec)
-        assert np.array_equal(got["b_res"].cpu().numpy().astype(np.uint32), want.b_res)
+    names = ("b_lim", "b_res", "limiter", "warps")
+
+    def check(got, want):
+        for name in names:
+            assert np.array_equal(got[name].cpu().numpy().astype(np.uint32), getattr(want, name)), name
+        assert np.array_equal(got["occ"].cpu().numpy().view(np.uint32), want.occ.view(np.uint32))
+        assert np.array_equal(got["occ_theo"].cpu().numpy().view(np.uint32), want.occ_theo.view(np.uint32))
         assert np.array_equal(to_np_u32(got["phi"]), want.phi)
+        assert int(got["n_unlaunchable"].item()) == want.n_unlaunchable
+
+    src = (lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block)
+    for n in (1, 3, 4, 5, 1023, 1024, 1025, 1026):
+        # offset by one element: no column is 16-byte aligned -> the scalar kernel, whatever n is
+        cols = [torch.from_numpy(np.ascontiguousarray(x[:n + 1]).view(np.int32)).cuda()[1:] for x in src]
+        assert all(c.data_ptr() % 16 == 4 for c in cols)
+        check(rm.occupancy(*cols, lib.spec), oracle.occupancy(*(x[1:n + 1] for x in src), lib.spec))
+        # aligned columns, ragged n: 128-bit loads, a scalar tail, and phi rows that are aligned or not by n
+        cols = [torch.from_numpy(np.ascontiguousarray(x[:n]).view(np.int32)).cuda() for x in src]
+        assert all(c.data_ptr() % 16 == 0 for c in cols)
+        check(rm.occupancy(*cols, lib.spec), oracle.occupancy(*(x[:n] for x in src), lib.spec))
     empty = rm.occupancy([], [], [], [], lib.spec)
     assert empty["occ"].numel() == 0
 
@@ -236,7 +247,8 @@ def test_pair_matrix_ranges_and_batching(rm, oracle):
 
 def test_config3_full_size(rm, oracle):
     """The headline workload in the launch configuration the benchmark times: full 512-profile matrix
-    at the base setting against the oracle, every entry; the greedy setting on a band of pairs."""
+    at the base setting and at the greedy setting (8 x 8 alignments, start filter, median) against the oracle,
+    every one of the 512 x 512 entries and the evaluation counts."""
     lib = rs.make_library(3)
     ol, gl = build_both(rm, oracle, lib)
     assert gl.status_flags() == 0
@@ -246,11 +258,14 @@ def test_config3_full_size(rm, oracle):
     got, ev = rm.pair_matrix(gl, mode=0, n_align=1, start_filter=0)
     assert int(ev.item()) == want_ev
     assert_close(got.cpu().numpy(), want)
-    # greedy setting: pairs 40 000 .. 40 600 of the triangle
-    import torch
+    # greedy setting on a band of pairs first (fast to localise a failure), then on every pair
     lo, hi = 40000, 40600
     wantg, wev = oracle.pair_matrix(ol, mode=0, n_align=8, start_filter=1, pair_begin=lo, pair_end=hi)
     gotg, gev = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1, pair_begin=lo, pair_end=hi)
+    assert int(gev.item()) == wev
+    assert_close(gotg.cpu().numpy(), wantg)
+    wantg, wev = oracle.pair_matrix(ol, mode=0, n_align=8, start_filter=1)
+    gotg, gev = rm.pair_matrix(gl, mode=0, n_align=8, start_filter=1)
     assert int(gev.item()) == wev
     assert_close(gotg.cpu().numpy(), wantg)
     assert gl.status_flags() == 0
@@ -315,9 +330,11 @@ def test_placement_end_to_end(rm, oracle, cfg):
     want = oracle.place(Po.astype(np.float32), cl.num_gpus, cl.max_residents, cl.ids, cl.expiry, cl.count, 0,
                         cl.arr_id, cl.arr_life, cl.lam)
     diff = np.nonzero(gpu != want.gpu)[0]
-    if diff.size:
-        assert want.near_tie[diff[0]], f"first mismatch at arrival {diff[0]} is not a near-tie"
-    print(f"\n[placement cfg{cfg}] mismatching decisions before divergence: {0 if not diff.size else 1}")
+    # expected: no mismatch at all.  The one documented exception is a decision the oracle's double shadow marks as
+    # a near-tie (two candidates, or a candidate and lambda, within 1e-5 relative): float rounding of the matrix may
+    # flip it, and the states diverge from there on.  Neither configuration has one.
+    assert diff.size == 0, (f"{diff.size} decisions differ, first at arrival {diff[0]} "
+                            f"(near-tie in the oracle's double shadow: {bool(want.near_tie[diff[0]])})")
 
 
 def test_placement_edge_cases(rm, oracle):
