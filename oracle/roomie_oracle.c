@@ -203,16 +203,26 @@ static void walk(const prof_view *A, const prof_view *B, uint32_t si, uint32_t s
  * kernels took beyond their isolated durations; the run ends when either
  * model has completed its last kernel.
  *
+ * Time is in integer ticks here as everywhere else, so that the order of
+ * events (which kernel completes first, which one started earlier) is a
+ * matter of integers and not of floating-point rounding.  The work of a
+ * kernel is counted in block-ticks: d_k * b in all; in one tick a kernel
+ * running with b~ blocks does b~ of them, so it completes after
+ * ceil(work left / b~) ticks (its last tick may be only partly used) and a
+ * kernel that keeps all its blocks takes exactly d_k.  A tick in which a
+ * kernel runs with b~ of its b blocks delays it by (b - b~) / b.
+ *
  * Policies for b~ (the paper names them, it does not spell them out):
  *   2 EQUAL    each kernel may use half of every SM resource;
  *   3 PRIORITY model i's kernel keeps its blocks, model j's kernel gets what
  *              is left of every resource;
  *   4 FCFS     the same with priority to the kernel that started earlier
  *              (model i on a tie).
- * A kernel left without a single block waits (rate 0) while the other runs
- * at full occupancy; under EQUAL, when neither fits into half an SM, the
- * kernel that started earlier (model i on a tie) runs alone.
- * Per-block demands come from phi at the resident block count b.
+ * A kernel left without a single block waits while the other runs at full
+ * occupancy; under EQUAL, when neither fits into half an SM, the kernel
+ * that started earlier (model i on a tie) runs alone.
+ * Per-block demands come from phi at the resident block count b.  A kernel
+ * without a resident block (b = 0) never interferes and takes d_k.
  * ------------------------------------------------------------------ */
 typedef struct { uint64_t wb, regs, smem, b; } block_need;
 
@@ -237,71 +247,84 @@ static uint64_t blocks_in(const block_need *n, uint64_t warps, uint64_t regs, ui
     return b;
 }
 
+/* one model during the co-run */
+typedef struct {
+    const prof_view *p;
+    uint32_t k;        /* its active kernel, or the next one while it idles              */
+    uint64_t b;        /* blocks that kernel runs with alone (1 stands in for b = 0)     */
+    uint64_t left;     /* work left, block-ticks                                         */
+    uint64_t idle;     /* ticks of gap left before kernel k starts                       */
+    uint64_t began;    /* tick at which kernel k started                                 */
+    double delay;      /* ticks lost so far                                              */
+} corun;
+
+static void corun_start_kernel(corun *m, uint64_t now)
+{
+    const uint64_t b = m->p->phi[3 * m->p->phi_stride + m->k];
+    m->b = b ? b : 1;
+    m->left = (uint64_t)m->p->dt[m->k] * m->b;
+    if (m->idle == 0) m->began = now;
+}
+
 static void walk_detailed(const prof_view *A, const prof_view *B, uint32_t si, uint32_t sj,
                           const uint64_t cap[4], int policy,
                           double *delta_i, double *delta_j, uint64_t *V, uint64_t *evals)
 {
-    uint32_t k[2] = { si, sj };
-    const prof_view *M[2] = { A, B };
-    double work[2], gap[2] = { 0.0, 0.0 }, began[2] = { 0.0, 0.0 }, lost[2] = { 0.0, 0.0 };
-    double now = 0.0, both = 0.0;
-    uint64_t ev = 0;
-    work[0] = A->dt[si]; work[1] = B->dt[sj];
-    while (k[0] < A->q && k[1] < B->q) {
+    corun M[2];
+    uint64_t now = 0, ev = 0;
+    memset(M, 0, sizeof(M));
+    M[0].p = A; M[0].k = si; M[1].p = B; M[1].k = sj;
+    corun_start_kernel(&M[0], 0);
+    corun_start_kernel(&M[1], 0);
+    while (M[0].k < A->q && M[1].k < B->q) {
         ++ev;
-        double rate[2] = { 1.0, 1.0 };
-        const int active0 = gap[0] <= 0.0, active1 = gap[1] <= 0.0;
-        int contend = 0;
-        if (active0 && active1 && A->phi[k[0]] > 0 && B->phi[k[1]] > 0 && interferes(A, k[0], B, k[1], cap)) {
-            const block_need n0 = need_of(A, k[0]), n1 = need_of(B, k[1]);
-            uint64_t b0, b1;
-            contend = 1;
+        /* blocks each active kernel runs with until the next event */
+        uint64_t bt[2] = { M[0].b, M[1].b };
+        if (M[0].idle == 0 && M[1].idle == 0 && A->phi[M[0].k] > 0 && B->phi[M[1].k] > 0 &&
+            interferes(A, M[0].k, B, M[1].k, cap)) {
+            const block_need n0 = need_of(A, M[0].k), n1 = need_of(B, M[1].k);
             if (policy == 2) {
-                b0 = blocks_in(&n0, cap[0] / 2, cap[1] / 2, cap[2] / 2, cap[3] / 2);
-                b1 = blocks_in(&n1, cap[0] / 2, cap[1] / 2, cap[2] / 2, cap[3] / 2);
-                if (b0 == 0 && b1 == 0) { if (began[0] <= began[1]) b0 = n0.b; else b1 = n1.b; }
-                else if (b0 == 0) b1 = n1.b;
-                else if (b1 == 0) b0 = n0.b;
+                bt[0] = blocks_in(&n0, cap[0] / 2, cap[1] / 2, cap[2] / 2, cap[3] / 2);
+                bt[1] = blocks_in(&n1, cap[0] / 2, cap[1] / 2, cap[2] / 2, cap[3] / 2);
+                if (bt[0] == 0 && bt[1] == 0) { if (M[0].began <= M[1].began) bt[0] = n0.b; else bt[1] = n1.b; }
+                else if (bt[0] == 0) bt[1] = n1.b;
+                else if (bt[1] == 0) bt[0] = n0.b;
             } else {
-                const int first = (policy == 3 || began[0] <= began[1]) ? 0 : 1;
+                const int first = (policy == 3 || M[0].began <= M[1].began) ? 0 : 1;
                 const block_need *hi = first == 0 ? &n0 : &n1, *lo = first == 0 ? &n1 : &n0;
-                const uint64_t bl = blocks_in(lo, cap[0] - hi->wb * hi->b, cap[1] - hi->regs * hi->b,
-                                              cap[2] - hi->smem * hi->b, cap[3] - hi->b);
-                b0 = first == 0 ? n0.b : bl;
-                b1 = first == 0 ? bl : n1.b;
+                bt[1 - first] = blocks_in(lo, cap[0] - hi->wb * hi->b, cap[1] - hi->regs * hi->b,
+                                          cap[2] - hi->smem * hi->b, cap[3] - hi->b);
             }
-            rate[0] = (double)b0 / (double)n0.b;
-            rate[1] = (double)b1 / (double)n1.b;
         }
-        /* time to the next event: a kernel completes or a gap ends */
-        double t[2];
-        for (int m = 0; m < 2; ++m)
-            t[m] = gap[m] > 0.0 ? gap[m] : (rate[m] > 0.0 ? work[m] / rate[m] : INFINITY);
-        const double dt = t[0] < t[1] ? t[0] : t[1];
-        now += dt;
-        if (contend) both += dt;
+        /* ticks to the next event: a gap ends or a kernel completes */
+        uint64_t until[2], step = UINT64_MAX;
         for (int m = 0; m < 2; ++m) {
-            if (gap[m] > 0.0) {
-                gap[m] = t[m] <= dt ? 0.0 : gap[m] - dt;
-                if (gap[m] <= 0.0) began[m] = now;
+            until[m] = M[m].idle > 0 ? M[m].idle
+                     : bt[m] > 0 ? (M[m].left + bt[m] - 1) / bt[m] : UINT64_MAX;
+            if (until[m] < step) step = until[m];
+        }
+        if (step == UINT64_MAX) break;                          /* cannot happen: one of the two always runs */
+        now += step;
+        for (int m = 0; m < 2; ++m) {
+            corun *c = &M[m];
+            if (c->idle > 0) {
+                c->idle -= step;
+                if (c->idle == 0) c->began = now;
                 continue;
             }
-            lost[m] += dt * (1.0 - rate[m]);
-            if (t[m] <= dt) {                                   /* this kernel completes */
-                const prof_view *p = M[m];
-                const uint32_t done = k[m]++;
-                if (k[m] < p->q) {
-                    gap[m] = (double)p->start[k[m]] - ((double)p->start[done] + (double)p->dt[done]);
-                    work[m] = p->dt[k[m]];
-                    if (gap[m] <= 0.0) { gap[m] = 0.0; began[m] = now; }
+            c->delay += (double)(step * (c->b - bt[m])) / (double)c->b;
+            if (until[m] == step) {                                /* this kernel completes */
+                const uint32_t done = c->k++;
+                if (c->k < c->p->q) {
+                    c->idle = (uint64_t)c->p->start[c->k] - ((uint64_t)c->p->start[done] + c->p->dt[done]);
+                    corun_start_kernel(c, now);
                 }
             } else {
-                work[m] -= dt * rate[m];
+                c->left -= step * bt[m];
             }
         }
     }
-    (void)both;
-    *delta_i = lost[0]; *delta_j = lost[1]; *V = 0; *evals = ev;   /* V is not defined in this mode */
+    *delta_i = M[0].delay; *delta_j = M[1].delay; *V = 0; *evals = ev;   /* V is not defined in this mode */
 }
 
 static int cmp_double(const void *x, const void *y)

@@ -1,5 +1,6 @@
 """Pins for the oracle's Section 3.2 simulator (adjusted occupancy, two-phase execution, partition policies):
-the paper's two-phase formula on hand cases, closed forms per policy, and an independent unit-step integrator."""
+the paper's two-phase formula on hand cases, closed forms per policy and per rate, and an independent tick-by-tick
+integrator (exact rationals, no event logic) at every rate b~/b the policies produce."""
 from fractions import Fraction
 
 import numpy as np
@@ -78,9 +79,11 @@ def test_no_interference_and_gaps(oracle):
 
 
 # ---------------------------------------------------------------------------------------
-# independent unit-step integrator: the kernel kinds below only produce rates 0, 1/2 and 1 and all
-# durations and gaps are multiples of 1024 ticks, so every event falls on an integer tick and a
-# one-tick stepper is exact
+# independent tick-by-tick integrator.  It knows nothing of events: every tick it looks at the two active
+# kernels, decides how many blocks each runs with, and moves each forward by one tick's worth of work (exact
+# rationals).  A kernel is complete at the first tick boundary at which its work is used up; its successor (or
+# the gap before it) starts there.  That is the simulator's definition, whatever b~/b is, so no restriction on
+# durations or rates is needed.
 # ---------------------------------------------------------------------------------------
 def stepper(ol, a, b, si, sj, policy):
     cap = [ol.spec.threads_per_sm // 32, ol.spec.regs_per_sm, ol.spec.smem_per_sm, ol.spec.blocks_per_sm]
@@ -92,6 +95,7 @@ def stepper(ol, a, b, si, sj, policy):
                     gap=0, began=0, lost=Fraction(0))
     M = [load(a, si), load(b, sj)]
     t = 0
+    rates = set()
     while M[0]["k"] < M[0]["q"] and M[1]["k"] < M[1]["q"]:
         rate = [Fraction(1), Fraction(1)]
         if M[0]["gap"] == 0 and M[1]["gap"] == 0:
@@ -118,6 +122,7 @@ def stepper(ol, a, b, si, sj, policy):
                     bt[first] = nb[first]
                     bt[other] = fit(other, left)
                 rate = [Fraction(bt[m], nb[m]) for m in range(2)]
+                rates.update(rate)
         t += 1
         for i, m in enumerate(M):
             if m["gap"] > 0:
@@ -135,7 +140,7 @@ def stepper(ol, a, b, si, sj, policy):
                     m["work"] = Fraction(int(m["dt"][m["k"]]))
                     if m["gap"] == 0:
                         m["began"] = t
-    return M[0]["lost"], M[1]["lost"]
+    return M[0]["lost"], M[1]["lost"], rates
 
 
 @pytest.mark.parametrize("seed", range(4))
@@ -152,11 +157,85 @@ def test_against_unit_step_integrator(oracle, seed):
     for policy in (EQUAL, PRIORITY, FCFS):
         d = oracle.pair(ol, 0, 1, mode=policy, n_align=0)
         for c in range(d.kept):
-            li, lj = stepper(ol, 0, 1, int(d.s_i[c]), int(d.s_j[c]), policy)
+            li, lj, _ = stepper(ol, 0, 1, int(d.s_i[c]), int(d.s_j[c]), policy)
             assert d.delta_i[c] == pytest.approx(float(li), abs=1e-9), (policy, c)
             assert d.delta_j[c] == pytest.approx(float(lj), abs=1e-9), (policy, c)
             hits += li > 0 or lj > 0
     assert hits > 0
+
+
+# kernel kinds on the cloud SM (65536 registers, 64 warps) whose partitions give every rate of the common case:
+#   HEAVY  4 blocks x 16384 registers      THREE  the same kernel, 3 blocks resident (grid of 324 on 108 SMs)
+#   HALF   2 such blocks                   ONE    1 such block
+#   TRIO   3 blocks x 20480 registers (256 threads x 80 registers)
+# PRIORITY / FCFS: beside HALF, HEAVY keeps 2 of 4 (1/2) and TRIO 1 of 3 (1/3); beside ONE, HEAVY keeps 3 of 4
+# (3/4) and TRIO 2 of 3 (2/3); beside THREE, HEAVY keeps 1 of 4 (1/4), TRIO none (it waits).
+# EQUAL (32768 registers each): HEAVY 2 of 4, TRIO 1 of 3, THREE 2 of 3, HALF and ONE untouched.
+THREE = (256, 64, 0, 324)
+ONE = (256, 64, 0, 100)
+TRIO = (256, 80, 0, 10000)
+LIGHT = (64, 0, 0, 100)
+SMEM5 = (128, 0, 81920, 10000)            # 2 blocks by shared memory; two of them never fit together
+
+
+def test_general_rates_hand_cases(oracle):
+    """One kernel against one kernel, durations in whole ticks: d_i = 12 ticks, d_j = 36 ticks, model i first."""
+    t = 0.001                                                       # one tick in microseconds
+
+    def run(ki, kj, policy, di=12, dj=36):
+        d, _ = sim(oracle, [[ki + (di * t, 0.0)], [kj + (dj * t, 0.0)]], policy)
+        return d.delta_i[0], d.delta_j[0]
+    # PRIORITY: i untouched for its 12 ticks; j runs at rate r meanwhile and loses 12 (1 - r)
+    assert run(ONE, HEAVY, PRIORITY) == (0.0, pytest.approx(3.0))       # r = 3/4
+    assert run(ONE, TRIO, PRIORITY) == (0.0, pytest.approx(4.0))        # r = 2/3
+    assert run(HALF, TRIO, PRIORITY) == (0.0, pytest.approx(8.0))       # r = 1/3
+    assert run(THREE, HEAVY, PRIORITY) == (0.0, pytest.approx(9.0))     # r = 1/4
+    assert run(THREE, TRIO, PRIORITY) == (0.0, pytest.approx(12.0))     # r = 0: j waits for all 12 ticks
+    # EQUAL: THREE keeps 2 of 3 blocks (12 ticks of work take 18), HEAVY 2 of 4 meanwhile (loses 18 / 2)
+    assert run(THREE, HEAVY, EQUAL) == (pytest.approx(6.0), pytest.approx(9.0))
+    # a duration that the rate does not divide: 10 ticks of work at 3/4 take ceil(40 / 3) = 14 whole ticks;
+    # j (priority to i = ONE with 20 ticks) runs 14 ticks at 3/4 and loses 14 / 4
+    assert run(ONE, HEAVY, PRIORITY, di=20, dj=10) == (0.0, pytest.approx(3.5))
+
+
+def _random_general_profiles(seed):
+    rng = np.random.default_rng(100 + seed)
+    kinds = [HEAVY, HALF, THREE, ONE, TRIO, LIGHT, SMEM5]
+    t = 0.001
+    profs = []
+    for _ in range(2):
+        q = int(rng.integers(2, 8))
+        profs.append([kinds[int(rng.integers(0, len(kinds)))] +
+                      (t * int(rng.integers(1, 90)), t * int(rng.integers(0, 3)) * int(rng.integers(0, 25)))
+                      for _ in range(q)])
+    return profs
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_general_rates_against_tick_integrator(oracle, seed):
+    """Random short profiles of the kinds above with arbitrary whole-tick durations and gaps, every alignment,
+    every policy, against the tick-by-tick integrator."""
+    ol = oracle.library_build(make_lib(_random_general_profiles(seed)))
+    for policy in (EQUAL, PRIORITY, FCFS):
+        for a, b in ((0, 1), (1, 0), (0, 0)):
+            d = oracle.pair(ol, a, b, mode=policy, n_align=0)
+            for c in range(d.kept):
+                li, lj, _ = stepper(ol, a, b, int(d.s_i[c]), int(d.s_j[c]), policy)
+                assert d.delta_i[c] == pytest.approx(float(li), rel=1e-12, abs=1e-12), (policy, a, b, c)
+                assert d.delta_j[c] == pytest.approx(float(lj), rel=1e-12, abs=1e-12), (policy, a, b, c)
+
+
+def test_general_rate_cases_cover_every_rate(oracle):
+    """The random cases above are only a pin at general rates if those rates occur in them."""
+    seen = set()
+    for seed in range(8):
+        ol = oracle.library_build(make_lib(_random_general_profiles(seed)))
+        for policy in (EQUAL, PRIORITY, FCFS):
+            for a, b in ((0, 1), (1, 0)):
+                for si, sj in ((0, 0), (1, 0), (0, 1), (1, 1)):
+                    seen |= stepper(ol, a, b, si, sj, policy)[2]
+    want = {Fraction(0), Fraction(1, 4), Fraction(1, 3), Fraction(1, 2), Fraction(2, 3), Fraction(3, 4), Fraction(1)}
+    assert want <= seen, sorted(want - seen)
 
 
 def test_detailed_is_at_least_as_pessimistic_as_waiting_never(oracle):
