@@ -12,8 +12,11 @@
  *
  * General conventions
  *   - Every data pointer is a DEVICE pointer owned by the caller unless its comment says
- *     "host".  The library never allocates or frees memory and keeps no pointer after a call
- *     returns; scratch space is passed in as `workspace`.
+ *     "host".  The library never allocates or frees device memory and keeps no pointer after a
+ *     call returns; scratch space is passed in as `workspace`.  Two documented exceptions:
+ *     roomie_pair_interference_static works in a fixed array inside the library image instead
+ *     of a workspace, and roomie_profile_enable creates CUDA events (host-side objects).  On the
+ *     host, the size arithmetic of the pair calls keeps two small per-thread vectors.
  *   - Calls only enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default
  *     stream) and return without synchronising, except where a comment says otherwise.
  *   - Return value: ROOMIE_OK or a negative roomie_status.  Data-dependent conditions
@@ -144,9 +147,13 @@ int roomie_library_build(const roomie_library *lib /* host */, const roomie_kern
  *   EQUAL    each of the two kernels may use half of every SM resource;
  *   PRIORITY the kernel of the pair's first model keeps its blocks, the other gets the remainder;
  *   FCFS     the same with priority to the kernel that started earlier (first model on a tie).
+ * Time is in whole ticks here too: the work of a kernel is d_k * b block-ticks, a kernel running with
+ * b~ blocks does b~ of them per tick and completes after ceil(work left / b~) ticks, and a tick spent
+ * with b~ of b blocks delays it by (b - b~)/b; so which kernel completes first, and which started
+ * earlier, never depends on rounding.
  * The alignment set, median, gamma and /T are applied as for the other modes; V is 0 and `evals`
- * counts simulation events.  With PRIORITY, P[a][b] and P[b][a] of an unordered pair both come from
- * the walk in which the lower-numbered profile has priority. */
+ * counts simulation events (a gap ends or a kernel completes).  With PRIORITY, P[a][b] and P[b][a] of
+ * an unordered pair both come from the walk in which the lower-numbered profile has priority. */
 #define ROOMIE_WALK_DETAILED_EQUAL 2
 #define ROOMIE_WALK_DETAILED_PRIORITY 3
 #define ROOMIE_WALK_DETAILED_FCFS 4
@@ -161,7 +168,9 @@ typedef struct roomie_opts {
                                at most 4096 alignments per pair                                  */
     int32_t start_filter;   /* 1: keep only alignments whose two start kernels interfere (Eq. 2) */
     float lambda;           /* degradation budget of Algorithm 2 (the paper uses 0.5)            */
-    uint32_t max_residents; /* slots per GPU in the cluster state                                */
+    uint32_t max_residents; /* placement calls: 0, or the slot count of the cluster state they are
+                               given (anything else is ROOMIE_ERR_INVALID_ARG); the state's own
+                               max_residents is what counts                                       */
     int32_t admit_rule;     /* ROOMIE_ADMIT_*: which quantity must stay below lambda             */
     int32_t objective;      /* ROOMIE_OBJECTIVE_*: which quantity the chosen GPU minimises       */
 } roomie_opts;
@@ -267,7 +276,8 @@ int roomie_multi_estimate(const float *Pmat, uint32_t P, const int32_t *resident
 /* Cluster state, updated in place by roomie_place (host struct of device arrays). */
 typedef struct roomie_cluster_state {
     uint32_t num_gpus;      /* G <= 1024                                                     */
-    uint32_t max_residents; /* R <= 64 slots per GPU                                         */
+    uint32_t max_residents; /* R <= 64 slots per GPU, and G * R <= 8192 (the state of one
+                               stream lives in one SM's shared memory)                       */
     int32_t *ids;           /* [G*R] profile id per slot, residents packed first, -1 = free  */
     uint32_t *expiry;       /* [G*R] arrival tick at which the resident leaves, 0 = never    */
     uint32_t *count;        /* [G] residents per GPU                                         */
@@ -285,7 +295,12 @@ typedef struct roomie_cluster_state {
  *   (optional) predicted drop of the arriving model there.
  * Decisions are taken in float32 with the fixed summation order of roomie_multi_estimate;
  * opts->admit_rule and opts->objective select the variants described at roomie_opts.
- * Errors: INVALID_ARG, CUDA. */
+ * Profile ids are checked on the device, where they live: an arrival whose id is outside [0, P) is
+ * not placed and gets gpu_out = ROOMIE_PLACE_BAD_ID (the state is left as it was); a cluster state
+ * that holds such an id among its residents makes every arrival of the call come back that way.
+ * Errors: INVALID_ARG (shape limits above, unknown rule or objective, opts->max_residents that
+ * contradicts the state), CUDA. */
+#define ROOMIE_PLACE_BAD_ID (-2)
 int roomie_place(const float *Pmat, uint32_t P, const roomie_cluster_state *state /* host struct */,
                  const int32_t *arr_id, const uint32_t *arr_life, uint32_t n, const roomie_opts *opts /* host */,
                  int32_t *gpu_out, float *mean_out, float *mu_arr_out, void *stream);

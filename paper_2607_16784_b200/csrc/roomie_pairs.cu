@@ -239,8 +239,6 @@ constexpr int kTileLoad = kTileItems + 2;                               // one l
 constexpr int kTopIndex = kTileLoad + kChunk;                           // unified indices stay below this
 constexpr int kRecSlots = kTopIndex + (kTopIndex >> kPadShift) + 1;
 constexpr int kTileCtasPerSm = 8;
-constexpr unsigned long long kWaitNs = 1000000000ull;                    // bound of every wait on a copy: 1 s
-constexpr uint32_t kWaitSpins = 1u << 24;
 
 template <bool kWithV>
 __device__ __forceinline__ void block_reduce_store(float di, float dj, unsigned long long V, uint32_t ties,
@@ -269,42 +267,7 @@ __device__ __forceinline__ float small_int_to_float(uint32_t v) {
     return __uint_as_float(0x4B000000u | v) - 8388608.0f;
 }
 
-// ---- asynchronous staging: mbarrier + bulk copies ---------------------------------------
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-}
-// one arrival that also announces `bytes` of copies that will complete on the barrier
-__device__ __forceinline__ void mbar_arrive_expect(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// waits for the phase with the given parity; gives up after kWaitNs (and, should the timer not
-// advance, after kWaitSpins polls)
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, unsigned long long limit_ns = kWaitNs) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (uint32_t spin = 0; spin < kWaitSpins; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (global_ns() - t0 > limit_ns) return false;
-    }
-    return false;
-}
+// ---- asynchronous staging: bulk copies that complete on an mbarrier (helpers in roomie_common.cuh) ----
 // bytes: a multiple of 16; both addresses 16-byte aligned
 __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -640,6 +603,7 @@ static void pair_of_host(uint64_t p, uint32_t P, uint32_t& a, uint32_t& b) {
 static uint32_t host_grid_count(uint32_t q, uint32_t A) { return (A == 0 || A > q) ? q : A; }
 
 struct Need { uint64_t walks, tiles; };
+constexpr uint64_t kDetailedExtraTiles = 160;     // 5 KB: the 1026-word bucket table of the walk sort
 
 // upper bound of walk slots and tiles for pairs [p0, p1): a walk of a pair has at most
 // q_a + q_b - 1 steps whatever its alignment.  Short ranges are counted pair by pair; long ones row by
@@ -691,6 +655,7 @@ static bool batch_need(const roomie_library* lib, const roomie_opts* o, bool exp
         }
     }
     need.walks = (explicit_pair ? 1 : (p1 - p0)) * (uint64_t)slots;
+    if (detailed) tiles = need.walks + kDetailedExtraTiles;       // one result per walk slot + the sort's bucket table
     need.tiles = tiles;
     return true;
 }
@@ -776,12 +741,48 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
     lv.cap = make_cap(lib->spec);
 
     if (o->walk_mode >= ROOMIE_WALK_DETAILED_EQUAL) {
-        // Section 3.2 simulator: one thread per walk writes its result where the tile partials go
+        // Section 3.2 simulator: the walks are sorted by expected length (plan, scan, scatter), then persistent
+        // lanes pull them; every walk writes its result where the tile partials go.  The sort's scratch lives in
+        // the tile-descriptor area: 32 bytes per walk plus kDetailedExtraTiles descriptors are reserved, 22 bytes
+        // per walk and the bucket table are used.
+        unsigned char* area = reinterpret_cast<unsigned char*>(tiles);
         DetailedArgs da;
         da.lib = lv; da.ps = ps; da.slots = slots; da.n_align = o->n_align; da.start_filter = o->start_filter;
-        da.policy = o->walk_mode; da.spec = lib->spec; da.walks = walks; da.partials = partials;
+        da.spec = lib->spec; da.walks = walks; da.partials = partials; da.status = lib->status;
+        da.seeds = reinterpret_cast<WalkSeed*>(area);
+        da.order = reinterpret_cast<uint32_t*>(area + need.walks * sizeof(WalkSeed));
+        da.bucket = reinterpret_cast<uint16_t*>(area + need.walks * (sizeof(WalkSeed) + sizeof(uint32_t)));
+        da.hist = reinterpret_cast<uint32_t*>(area + ((need.walks * 22 + 15) & ~(uint64_t)15));
+        uint32_t qmax = 1;
+        if (ps.explicit_pair) {
+            const uint32_t* off = lib->offsets_host;
+            qmax = off[ps.a + 1] - off[ps.a];
+            if (off[ps.b + 1] - off[ps.b] > qmax) qmax = off[ps.b + 1] - off[ps.b];
+        } else {
+            for (uint32_t p = 0; p < lib->num_profiles; ++p)
+                if (lib->offsets_host[p + 1] - lib->offsets_host[p] > qmax) qmax = lib->offsets_host[p + 1] - lib->offsets_host[p];
+        }
+        da.shift = 0;
+        while (((2ull * qmax) >> da.shift) >= (uint64_t)kSortBuckets) ++da.shift;
+        ROOMIE_CUDA_OK(cudaMemsetAsync(da.hist, 0, (kSortBuckets + 2) * sizeof(uint32_t), st));
+        uint64_t pblocks = (need.walks + 255) / 256;
+        if (pblocks > (uint64_t)sm_count() * 8) pblocks = (uint64_t)sm_count() * 8;
+        detailed_plan_kernel<<<(unsigned)pblocks, 256, 0, st>>>(da);
+        note_launch();
+        detailed_scan_kernel<<<1, kSortBuckets, 0, st>>>(da.hist);
+        note_launch();
+        detailed_scatter_kernel<<<(unsigned)pblocks, 256, 0, st>>>(da);
+        note_launch();
+        ROOMIE_CUDA_OK(cudaGetLastError());
+        uint64_t wblocks = (need.walks + kDetailedThreads - 1) / kDetailedThreads;
+        if (wblocks > (uint64_t)sm_count() * 12) wblocks = (uint64_t)sm_count() * 12;
         profile_mark(st, true);
-        detailed_walk_kernel<<<(unsigned)((need.walks + 127) / 128), 128, 0, st>>>(da);
+        if (o->walk_mode == ROOMIE_WALK_DETAILED_EQUAL)
+            detailed_walk_kernel<ROOMIE_WALK_DETAILED_EQUAL><<<(unsigned)wblocks, kDetailedThreads, 0, st>>>(da);
+        else if (o->walk_mode == ROOMIE_WALK_DETAILED_PRIORITY)
+            detailed_walk_kernel<ROOMIE_WALK_DETAILED_PRIORITY><<<(unsigned)wblocks, kDetailedThreads, 0, st>>>(da);
+        else
+            detailed_walk_kernel<ROOMIE_WALK_DETAILED_FCFS><<<(unsigned)wblocks, kDetailedThreads, 0, st>>>(da);
         profile_mark(st, false);
         note_launch();
         ROOMIE_CUDA_OK(cudaGetLastError());

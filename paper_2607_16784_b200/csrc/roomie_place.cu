@@ -130,6 +130,21 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
     __syncthreads();
 
     const bool owner = tid < G;
+    {   // a resident id outside the matrix would send the reads below out of bounds: refuse the whole call
+        bool bad_id = false;
+        for (uint32_t i = tid; i < GR; i += blockDim.x) {
+            const uint32_t gpu = i / R, slot = i % R;
+            bad_id |= slot < min(g.count[gpu], R) && (uint32_t)g.ids[i] >= P;
+        }
+        if (__syncthreads_or(bad_id)) {
+            for (uint32_t i = tid; i < g.n; i += blockDim.x) {
+                g.gpu_out[i] = ROOMIE_PLACE_BAD_ID;
+                if (g.mean_out) g.mean_out[i] = 0.0f;
+                if (g.mu_arr_out) g.mu_arr_out[i] = 0.0f;
+            }
+            return;
+        }
+    }
     auto ID = [&](uint32_t t) -> int32_t& { return s_ids[t * G + tid]; };
     auto EX = [&](uint32_t t) -> uint32_t& { return s_exp[t * G + tid]; };
     auto PA = [&](uint32_t t) -> float& { return s_part[t * G + tid]; };
@@ -172,26 +187,28 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
         const uint32_t kn = min(kArrChunk, g.n - k0);
         __syncthreads();
         for (uint32_t i = tid; i < kn; i += blockDim.x) {
-            s_arr[i] = g.arr_id[k0 + i];
+            const int32_t id = g.arr_id[k0 + i];
+            s_arr[i] = (uint32_t)id < P ? id : -1;                     // -1: not a profile of this matrix
             s_arr[kArrChunk + i] = (int32_t)g.arr_life[k0 + i];
         }
         __syncthreads();
         if (g.matrix_mode == 1) {                                      // prime the ring: arrivals 0 and 1
-            prefetch(0, s_arr[0]);
+            prefetch(0, max(s_arr[0], 0));
             cp_async_commit();
-            if (kn > 1) prefetch(1, s_arr[1]);
+            if (kn > 1) prefetch(1, max(s_arr[1], 0));
             cp_async_commit();
             cp_async_wait<1>();                                        // arrival 0 landed
             __syncthreads();
         }
         for (uint32_t k = 0; k < kn; ++k) {
             const uint32_t now = tick0 + k0 + k;
-            const int32_t inc = s_arr[k];
+            const bool bad_arrival = s_arr[k] < 0;                      // scored by nobody, reported as such
+            const int32_t inc = max(s_arr[k], 0);
             const float *row_inc, *col_inc;
             uint32_t col_stride;
             if (g.matrix_mode == 1) {
                 // arrival k's row and column are in the ring (made visible by the last barrier)
-                if (k + 2 < kn) prefetch(k + 2, s_arr[k + 2]);
+                if (k + 2 < kn) prefetch(k + 2, max(s_arr[k + 2], 0));
                 cp_async_commit();
                 row_inc = s_mat + (size_t)(k % kRing) * 2 * P; col_inc = row_inc + P; col_stride = 1;
             } else if (g.matrix_mode == 0) {
@@ -226,7 +243,7 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
                     c = w;
                     recompute_partials(c);
                 }
-                if (c < R) {                                           // what-if: residents + the arrival
+                if (c < R && !bad_arrival) {                           // what-if: residents + the arrival
                     float tot = 0.0f, worst = 0.0f;
                     if constexpr (kSlots > 0) {
                         float to_inc[kSlots], from_inc[kSlots], part[kSlots];
@@ -277,7 +294,7 @@ __global__ void __launch_bounds__(1024) place_kernel(PlaceArgs g) {
             }
             if (best == kNoGpu) {
                 if (tid == 0) {
-                    g.gpu_out[k0 + k] = -1;
+                    g.gpu_out[k0 + k] = bad_arrival ? ROOMIE_PLACE_BAD_ID : -1;
                     if (g.mean_out) g.mean_out[k0 + k] = 0.0f;
                     if (g.mu_arr_out) g.mu_arr_out[k0 + k] = 0.0f;
                 }
@@ -390,6 +407,19 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
 
     const float* __restrict__ Pm = g.Pm;
 
+    {   // a resident id outside the matrix would send the reads below out of bounds: refuse the whole call
+        bool bad_id = false;
+        if (owner)
+            for (uint32_t p = 0; p < min(g.count[gpu], R); ++p) bad_id |= (uint32_t)g.ids[gpu * R + p] >= P;
+        if (__syncthreads_or(bad_id)) {
+            for (uint32_t i = tid; i < g.n; i += blockDim.x) {
+                g.gpu_out[i] = ROOMIE_PLACE_BAD_ID;
+                if (g.mean_out) g.mean_out[i] = 0.0f;
+                if (g.mu_arr_out) g.mu_arr_out[i] = 0.0f;
+            }
+            return;
+        }
+    }
     // initial state: residents occupy physical slots 0..c-1 in arrival order
     uint32_t c = 0, ord = 0, free_mask = (1u << R) - 1u, next_exp = 0xffffffffu;
     if (owner) {
@@ -419,7 +449,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
 
     // fetch warps: what arrival a (staged index a_local, global index a_global) will need
     auto issue = [&](uint32_t a_local, uint32_t a_global) {
-        const int32_t inc = smi[oARR + a_local];
+        const int32_t inc = max(smi[oARR + a_local], 0);  // an id outside the matrix is staged as -1 and scored by nobody
         const float* row = Pm + (size_t)inc * P;          // P[inc][*]
         const float* col = Pm + inc;                      // P[*][inc]
         if (has_gpu) {
@@ -437,7 +467,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
         if (wid == n_owner_warps && lane < 2 * kYoungD) {
             const uint32_t d = (lane >> 1) + 1, dir = lane & 1u;
             if (a_local >= d) {
-                const int32_t old = smi[oARR + a_local - d];
+                const int32_t old = max(smi[oARR + a_local - d], 0);
                 cp_async_4_s(sm_base + 4u * (oYOUNG + ((a_global & (kYoungRing - 1)) * kYoungD + (d - 1)) * 2 + dir),
                              dir == 0 ? col + (size_t)old * P : row + old);
             }
@@ -450,7 +480,9 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
         __syncthreads();
         for (uint32_t i = tid; i < kn + 2 * kLead; i += blockDim.x) {
             const long long gi = (long long)k0 + i - kLead;
-            smi[oARR + i] = (gi >= 0 && gi < (long long)g.n) ? g.arr_id[gi] : 0;
+            int32_t id = 0;
+            if (gi >= 0 && gi < (long long)g.n) { id = g.arr_id[gi]; if ((uint32_t)id >= P) id = -1; }
+            smi[oARR + i] = id;
         }
         for (uint32_t i = tid; i < kn; i += blockDim.x) smi[oLIFE + i] = (int32_t)g.arr_life[k0 + i];
         __syncthreads();
@@ -497,7 +529,8 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             const uint32_t young_k = oYOUNG + (kg & (kYoungRing - 1)) * kYoungD * 2;
             uint32_t key_hi = 0xffffffffu;
             float mean = 0.0f, mu_inc = 0.0f;
-            if (owner && c < R) {                                            // what-if: residents + the arrival
+            const bool bad_arrival = smi[oARR + kl] < 0;
+            if (owner && c < R && !bad_arrival) {                            // what-if: residents + the arrival
                 float tot = 0.0f, worst = 0.0f;
                 // two-stage pipeline over the residents: while resident t is summed, the terms of t + 1 are on
                 // their way and the birth index and cached partial sum of t + 2 are being read (past the end
@@ -559,7 +592,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             // results stay in shared memory until the chunk ends: a global store inside the loop would
             // have to complete before every barrier
             if (best == kNoGpu) {
-                if (tid == 0) { smi[oOUT + k] = -1; sm[oOUT + chunk + k] = 0.0f; sm[oOUT + 2 * chunk + k] = 0.0f; }
+                if (tid == 0) { smi[oOUT + k] = bad_arrival ? ROOMIE_PLACE_BAD_ID : -1; sm[oOUT + chunk + k] = 0.0f; sm[oOUT + 2 * chunk + k] = 0.0f; }
             } else if (owner && gpu == (uint32_t)(best & 0xffffffffu)) {
                 const uint32_t pn = __ffs(free_mask) - 1u;                   // the slot the what-if wrote for
                 free_mask &= ~(1u << pn);
@@ -629,6 +662,7 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
     if (!arr_id || !arr_life || !gpu_out) return ROOMIE_ERR_INVALID_ARG;
     if (opts->admit_rule < 0 || opts->admit_rule > 1 || opts->objective < 0 || opts->objective > 2)
         return ROOMIE_ERR_INVALID_ARG;
+    if (opts->max_residents != 0 && opts->max_residents != state->max_residents) return ROOMIE_ERR_INVALID_ARG;
     PlaceArgs a;
     a.admit_rule = opts->admit_rule; a.objective = opts->objective;
     a.Pm = Pmat; a.P = P; a.G = state->num_gpus; a.R = state->max_residents;

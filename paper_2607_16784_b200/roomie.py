@@ -264,9 +264,10 @@ def pair_matrix(lib: Library, *, mode=TIMELINE, n_align=1, start_filter=0, pair_
     return out, evals
 
 
-def _pair_outputs(dev, detail_capacity):
-    out2 = torch.zeros(2, dtype=torch.float32, device=dev)
-    evals = torch.zeros(1, dtype=torch.int64, device=dev)
+def _pair_outputs(dev, detail_capacity, out2=None):
+    if out2 is None:
+        out2 = torch.zeros(2, dtype=torch.float32, device=dev)
+    evals = None if detail_capacity < 0 else torch.zeros(1, dtype=torch.int64, device=dev)
     res = dict(P2=out2, evals=evals)
     det = None
     if detail_capacity > 0:
@@ -300,11 +301,13 @@ def pair_interference(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1,
 
 
 def pair_interference_static(lib: Library, a: int, b: int, *, mode=TIMELINE, n_align=1, start_filter=0,
-                             detail_capacity=0, stream=None):
+                             detail_capacity=0, out2=None, stream=None):
     """roomie_pair_interference_static: the same result computed in the library's built-in scratch
-    array - for callers that cannot allocate device memory.  Calls that overlap on the GPU race."""
+    array - for callers that cannot allocate device memory.  Calls that overlap on the GPU race.
+    With `out2` (float32 [2] device tensor) given and no detail requested, the binding itself creates no
+    tensor either: the evaluation count is then not returned."""
     o = _opts(mode, n_align, start_filter)
-    res, det = _pair_outputs(lib.records.device, detail_capacity)
+    res, det = _pair_outputs(lib.records.device, -1 if (out2 is not None and detail_capacity == 0) else detail_capacity, out2)
     _check(_dll.roomie_pair_interference_static(C.byref(lib.c), a, b, C.byref(o), _ptr(res["P2"]),
                                                 _ptr(res["evals"]), C.byref(det) if det is not None else None,
                                                 _stream(stream)), "roomie_pair_interference_static")

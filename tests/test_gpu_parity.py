@@ -374,6 +374,45 @@ def test_placement_edge_cases(rm, oracle):
     assert np.array_equal(gpu, want.gpu)
 
 
+def test_placement_rejects_ids_outside_the_matrix(rm, oracle):
+    """Profile ids live on the device, so they are checked there: an arrival with an id outside [0, P) is not placed
+    (gpu_out = -2) and changes nothing - the other decisions equal those of the stream without it; a cluster state that
+    already holds such an id makes the whole call come back with -2.  Both placement kernels."""
+    rng = np.random.default_rng(2)
+    P = 24
+    Pm = (rng.random((P, P)) * 0.2).astype(np.float32)
+    for G, R in ((64, 8), (6, 12)):                                   # fast kernel, generic kernel
+        n = 200
+        aid = rng.integers(0, P, n).astype(np.int32)
+        life = rng.integers(1, 40, n).astype(np.uint32)
+        bad = aid.copy()
+        bad[[5, 77, 199]] = [P, -3, 1 << 20]
+        st = rm.ClusterState(G, R, [-1] * (G * R), [0] * (G * R), [0] * G, 0)
+        gpu = rm.place(Pm, st, bad, life, 0.5)[0].cpu().numpy()
+        assert (gpu[[5, 77, 199]] == -2).all() and (np.delete(gpu, [5, 77, 199]) >= -1).all()
+        # the oracle on the same stream with the three arrivals taken out, ticks kept: model them as arrivals nobody
+        # can take (an empty cluster slot count of zero is not expressible, so compare against a run that defers them)
+        keep = np.ones(n, bool); keep[[5, 77, 199]] = False
+        ids, exp, cnt = [-1] * (G * R), [0] * (G * R), [0] * G
+        want_gpu = np.full(n, -2, np.int32)
+        tick = 0
+        start = 0
+        for stop in (5, 77, 199, n):                                  # segments between the rejected arrivals
+            if stop > start:
+                w = oracle.place(Pm, G, R, ids, exp, cnt, tick, aid[start:stop], life[start:stop], 0.5)
+                want_gpu[start:stop] = w.gpu
+                ids, exp, cnt = w.ids, w.expiry, w.count
+            tick = stop + 1                                           # the rejected arrival still takes its tick
+            start = stop + 1
+        assert np.array_equal(gpu, want_gpu)
+        # a resident id outside the matrix: nothing is placed, the state stays as given
+        ids0 = np.full(G * R, -1, np.int32); ids0[R] = P + 7
+        cnt0 = np.zeros(G, np.uint32); cnt0[1] = 1
+        st = rm.ClusterState(G, R, ids0, [0] * (G * R), cnt0, 0)
+        gpu = rm.place(Pm, st, aid, life, 0.5)[0].cpu().numpy()
+        assert (gpu == -2).all() and np.array_equal(st.ids.cpu().numpy(), ids0) and int(st.tick.item()) == 0
+
+
 # ----------------------------------------------------------------------------- placement variants, batches
 @pytest.mark.parametrize("cfg", [2, 4])
 @pytest.mark.parametrize("admit_rule,objective", [(1, 0), (0, 1), (0, 2), (1, 2)])

@@ -38,13 +38,37 @@ def test_static_scratch_entry_point_matches_workspace_entry_point():
                           lib.dur_us, lib.gap_us, lib.offsets, lib.spec)
     calls = [(3, 17, dict(mode=0, n_align=8, start_filter=1)),     # many walks, several tiles each
              (5, 5, dict(mode=0, n_align=1, start_filter=0)),      # one walk: far less scratch than the call before
-             (30, 2, dict(mode=1, n_align=4, start_filter=0))]
-    # two (here three) calls in a row on the shared array, each compared with the workspace variant
+             (30, 2, dict(mode=1, n_align=4, start_filter=0)),
+             (7, 21, dict(mode=3, n_align=4, start_filter=1)),     # Section 3.2 simulator: the scratch also holds its walk sort
+             (9, 4, dict(mode=2, n_align=2, start_filter=0))]
+    # warm both entry points once, so that what is measured below is the call and not the first-use set-up of
+    # the runtime (module loading) or of torch's caching allocator
+    rm.pair_interference_static(gl, 0, 1, detail_capacity=64, **calls[0][2])
+    rm.pair_interference(gl, 0, 1, detail_capacity=64, **calls[0][2])
+    torch.cuda.synchronize()
+    # several calls in a row on the shared array, each compared with the workspace variant
     for a, b, kw in calls:
+        out2 = torch.zeros(2, dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+        rm.pair_interference_static(gl, a, b, out2=out2, **kw)     # outputs given: the call itself gets no memory
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == held               # nothing from torch's allocator ...
+        assert torch.cuda.mem_get_info()[0] >= free                # ... and nothing from the driver
         got = rm.pair_interference_static(gl, a, b, detail_capacity=64, **kw)
         want = rm.pair_interference(gl, a, b, detail_capacity=64, **kw)
         same(got, want)
-        assert int(want["n_kept"].item()) > 0 and float(want["P2"][0]) > 0
+        assert torch.equal(out2, got["P2"])
+        assert int(want["n_kept"].item()) > 0 and float(want["P2"].max()) > 0    # (with priority the first model loses nothing)
+    # Algorithm 1 as printed over the full alignment set, with per-alignment detail (the variant that does need
+    # scratch): two short profiles so that the q_a x q_b alignments fit the array
+    small = rs.make_library(0)
+    gs = rm.library_build(small.grid_blocks, small.block_threads, small.regs_per_thread, small.smem_per_block,
+                          small.dur_us, small.gap_us, small.offsets, small.spec)
+    got = rm.pair_interference_static(gs, 0, 1, mode=1, n_align=0, detail_capacity=2500)
+    want = rm.pair_interference(gs, 0, 1, mode=1, n_align=0, detail_capacity=2500)
+    same(got, want)
+    assert int(want["n_kept"].item()) == 2500
     # the same call twice in a row gives the same bits
     a, b, kw = calls[0]
     first = rm.pair_interference_static(gl, a, b, detail_capacity=64, **kw)
