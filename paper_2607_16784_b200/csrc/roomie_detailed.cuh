@@ -18,12 +18,16 @@
 //   FCFS      the same with the kernel that started earlier in the first role (first model on a tie).
 //
 // A walk is a chain of dependent events, so the parallelism is across walks, and the cost of a warp is its
-// longest walk.  Three things keep the lanes busy: (1) the walks of a batch are put in descending order of
-// their expected length by a counting sort (plan -> scan -> scatter), so the 32 walks of a warp are alike and
-// the longest start first; (2) warps are persistent and every lane pulls its next walk from a shared counter
-// when it is done; (3) the record of each model's next kernel is already in registers when the active one
-// completes, work left is kept both in block-ticks and in ticks at full occupancy so that an undisturbed
-// kernel needs no division, and the divisions that remain go through reciprocals with an integer correction.
+// longest walk times the instructions of one pass over the event code.  What keeps that product down:
+// (1) the walks of a batch are put in descending order of their expected length by a counting sort (plan ->
+// scan -> scatter), so the 32 walks of a warp are alike and the longest start first; (2) warps are persistent
+// and every lane pulls its next walk from a shared counter when it is done; (3) what depends on a kernel alone
+// (its blocks, the demand of one block, the blocks that fit into half an SM) is worked out once per kernel
+// of the library into an 8-byte side record, not once per event; (4) the record and side record of each model's
+// next kernel are already in registers when the active one completes; (5) the event code is written without
+// data-dependent branches except "a kernel completed" (the partition, the time to the next event and the
+// bookkeeping of both models are selects), so the lanes of a warp execute it together instead of one after the
+// other; the one division an event needs goes through a reciprocal with an integer correction.
 
 constexpr int kSortBuckets = 1024;
 constexpr int kDetailedThreads = 128;
@@ -31,7 +35,13 @@ constexpr int kDetailedThreads = 128;
 struct WalkSeed {              // what a lane needs to start a walk, written by the plan kernel
     uint32_t recA, recB;       // global index of each model's first record of the alignment
     uint32_t nA, nB;           // records from there to the end of each sequence
+    uint32_t sideA, sideB;     // index of the first side record of each model
 };
+
+// Per-kernel side record (64 bits): bits 0-7 blocks the kernel runs with alone (1 stands in for a kernel without
+// a resident block: it never interferes and takes its isolated time), 8-15 blocks that fit into half an SM,
+// 16-23 warps of one block, 24-43 shared-memory bytes of one block, 44-61 registers of one block.
+struct SideRange { uint32_t first_record, count, first_side; };
 
 struct DetailedArgs {
     LibView lib;
@@ -47,7 +57,61 @@ struct DetailedArgs {
     uint32_t* hist;            // [kSortBuckets] counts, then cursors; [kSortBuckets] = kept walks; [+1] = next to hand out
     uint32_t shift;            // bucket = (nA + nB) >> shift, reversed
     uint32_t* status;          // library status word
+    unsigned long long* side;  // side records
+    SideRange range[2];        // which records have side records, and where (an explicit pair: its two profiles)
+    uint32_t n_ranges;
 };
+
+// ---- arithmetic helpers ---------------------------------------------------------------------------------
+// x / d for an exact multiple x < 2^22 of d >= 1: the approximate quotient is within 1/2 of the true one
+__device__ __forceinline__ uint32_t div_exact(uint32_t x, uint32_t d) {
+    return (uint32_t)__float2int_rn(__fdividef((float)x, (float)d));
+}
+// floor(x / d) for x < 2^23, d >= 1: approximate quotient, one correction step in integers
+__device__ __forceinline__ uint32_t div_floor(uint32_t x, uint32_t d) {
+    uint32_t q = (uint32_t)__fdividef((float)x, (float)d);
+    const int32_t r = (int32_t)x - (int32_t)(q * d);
+    q -= r < 0 ? 1u : 0u;
+    q += (r >= 0 && (uint32_t)r >= d) ? 1u : 0u;
+    return q;
+}
+// ceil(x / d) for x < 2^45, 1 <= d <= 255, with inv = the double nearest to 1/d: the product is within 2^-7 of
+// the quotient, so its integer part is at most one off
+__device__ __forceinline__ unsigned long long div_ceil(unsigned long long x, uint32_t d, double inv) {
+    long long q = __double2ll_rz(__dmul_rn(__ull2double_rn(x), inv));
+    long long r = (long long)x - q * (long long)d;
+    const bool low = r < 0, high = r >= (long long)d;
+    q += high ? 1 : (low ? -1 : 0);
+    r += low ? (long long)d : (high ? -(long long)d : 0);
+    return (unsigned long long)q + (r != 0 ? 1ull : 0ull);
+}
+
+__device__ __forceinline__ uint32_t side_blocks(unsigned long long s) { return (uint32_t)s & 255u; }
+__device__ __forceinline__ uint32_t side_half_fit(unsigned long long s) { return ((uint32_t)s >> 8) & 255u; }
+__device__ __forceinline__ uint32_t side_warps(unsigned long long s) { return ((uint32_t)s >> 16) & 255u; }
+__device__ __forceinline__ uint32_t side_smem(unsigned long long s) { return (uint32_t)(s >> 24) & ((1u << 20) - 1u); }
+__device__ __forceinline__ uint32_t side_regs(unsigned long long s) { return (uint32_t)(s >> 44) & ((1u << 18) - 1u); }
+
+// ---- side records: once per kernel of the library (or of the two profiles of an explicit pair) ---------------
+__global__ void __launch_bounds__(256) detailed_side_kernel(DetailedArgs g) {
+    const roomie_gpu_spec sp = g.spec;
+    for (uint32_t rg = 0; rg < g.n_ranges; ++rg) {
+        const SideRange R = g.range[rg];
+        for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < R.count; i += gridDim.x * blockDim.x) {
+            const uint4 rec = __ldg(&g.lib.records[R.first_record + i]);
+            const uint32_t blocks = rec.w >> 22, b = blocks ? blocks : 1u;
+            const uint32_t warps = rec.z >> kWarpShift, regs = rec.z & ((1u << kWarpShift) - 1u),
+                           smem = rec.w & ((1u << 22) - 1u);
+            const uint32_t wb = div_exact(warps, b), rb = div_exact(regs, b), sb = div_exact(smem, b);
+            uint32_t f = min(blocks, sp.blocks_per_sm / 2);
+            if (wb) f = min(f, div_floor(sp.threads_per_sm / 64u, wb));
+            if (rb) f = min(f, div_floor(sp.regs_per_sm / 2, rb));
+            if (sb) f = min(f, div_floor(sp.smem_per_sm / 2, sb));
+            g.side[R.first_side + i] = (unsigned long long)b | ((unsigned long long)f << 8) | ((unsigned long long)wb << 16) |
+                                       ((unsigned long long)sb << 24) | ((unsigned long long)rb << 44);
+        }
+    }
+}
 
 // ---- plan: which alignments are kept, where they start, how long they may get -----------------------------
 __global__ void __launch_bounds__(256) detailed_plan_kernel(DetailedArgs g) {
@@ -66,13 +130,17 @@ __global__ void __launch_bounds__(256) detailed_plan_kernel(DetailedArgs g) {
         const uint32_t ca = c / gb, cb = c % gb;
         bool keep = ca < ga;
         WalkSeed s;
-        s.recA = s.recB = s.nA = s.nB = 0;
+        s.recA = s.recB = s.nA = s.nB = s.sideA = s.sideB = 0;
         if (keep) {
             const uint32_t si = grid_start(qa, g.n_align, ca), sj = grid_start(qb, g.n_align, cb);
             s.recA = offa + si; s.recB = offb + sj; s.nA = qa - si; s.nB = qb - sj;
+            // side records: of the whole library (index = record index) or of the pair's two profiles
+            s.sideA = s.recA - g.range[0].first_record + g.range[0].first_side;
+            const SideRange& rb = g.range[g.n_ranges - 1];
+            s.sideB = s.recB - rb.first_record + rb.first_side;
             if (g.start_filter) {
-                const uint4 ra = __ldg(&g.lib.records[s.recA]), rb = __ldg(&g.lib.records[s.recB]);
-                keep = phi_exceeds(g.lib.cap.lo - ra.z, g.lib.cap.hi - ra.w, rb.z, rb.w);
+                const uint4 ra = __ldg(&g.lib.records[s.recA]), rb2 = __ldg(&g.lib.records[s.recB]);
+                keep = phi_exceeds(g.lib.cap.lo - ra.z, g.lib.cap.hi - ra.w, rb2.z, rb2.w);
             }
         }
         if (keep) {
@@ -124,119 +192,69 @@ __global__ void __launch_bounds__(256) detailed_scatter_kernel(DetailedArgs g) {
     }
 }
 
-// ---- arithmetic helpers ---------------------------------------------------------------------------------
-// x / d for an exact multiple x < 2^22 of d >= 1: the approximate quotient is within 1/2 of the true one
-__device__ __forceinline__ uint32_t div_exact(uint32_t x, uint32_t d) {
-    return (uint32_t)__float2int_rn(__fdividef((float)x, (float)d));
-}
-// floor(x / d) for x < 2^23, d >= 1: approximate quotient, one correction step in integers
-__device__ __forceinline__ uint32_t div_floor(uint32_t x, uint32_t d) {
-    uint32_t q = (uint32_t)__fdividef((float)x, (float)d);
-    const int32_t r = (int32_t)x - (int32_t)(q * d);
-    if (r < 0) --q;
-    else if ((uint32_t)r >= d) ++q;
-    return q;
-}
-// ceil(x / d) for x < 2^45, 1 <= d <= 255, with inv = the double nearest to 1/d: the product is within 2^-7 of
-// the quotient, so its integer part is at most one off
-__device__ __forceinline__ unsigned long long div_ceil(unsigned long long x, uint32_t d, double inv) {
-    long long q = __double2ll_rz(__dmul_rn(__ull2double_rn(x), inv));
-    long long r = (long long)x - q * (long long)d;
-    if (r < 0) { --q; r += d; }
-    else if (r >= (long long)d) { ++q; r -= d; }
-    return (unsigned long long)q + (r != 0 ? 1ull : 0ull);
-}
-
 // One model of the co-run.  The record holds phi at the resident block count: warps = bits 20.. of z, registers
 // = low bits of z, shared memory = low bits of w, block slots = bits 22.. of w.
 struct CoModel {
-    const uint4* at;            // record of the NEXT kernel to fetch
-    uint32_t more;              // records still to fetch from `at`
-    uint4 rec, ahead;           // active kernel; the one after it (valid while `pending`)
-    uint32_t pending;           // kernels after the active one, fetched or not
-    uint32_t b;                 // blocks of the active kernel alone, at least 1
-    uint32_t fit;               // EQUAL: blocks that fit into half an SM; else unused
-    uint32_t wb, rg, sm;        // PRIORITY / FCFS: warps, registers, shared memory of one block
-    uint32_t idle;              // ticks of gap before the active kernel starts
-    uint32_t full;              // ticks it still needs at full occupancy = ceil(left / b)
-    unsigned long long left;    // block-ticks left
-    unsigned long long began;   // tick at which it started
-    double lost;                // delay so far, ticks
-    bool alive;                 // the sequence is not exhausted
+    uint4 rec, ahead;                   // active kernel; the one after it (valid while `pending`)
+    unsigned long long side, side_ahead;
+    uint32_t next_rec, next_side;       // where the kernel after `ahead` is
+    uint32_t more;                      // records still to fetch
+    uint32_t pending;                   // kernels after the active one, fetched or not
+    uint32_t idle;                      // ticks of gap before the active kernel starts
+    unsigned long long left;            // block-ticks left
+    unsigned long long began;           // tick at which it started
+    double lost;                        // delay so far, ticks
+    bool alive;                         // the sequence is not exhausted
 };
 
-template <int kPolicy>
-__device__ __forceinline__ void start_kernel(CoModel& m, const roomie_gpu_spec& sp, unsigned long long now) {
-    const uint32_t blocks = m.rec.w >> 22;
-    m.b = blocks ? blocks : 1u;
-    m.full = m.rec.y - m.rec.x;
-    m.left = (unsigned long long)m.full * m.b;
-    if (m.idle == 0) m.began = now;
-    const uint32_t warps = m.rec.z >> kWarpShift, regs = m.rec.z & ((1u << kWarpShift) - 1u),
-                   smem = m.rec.w & ((1u << 22) - 1u);
-    const uint32_t wb = div_exact(warps, m.b), rg = div_exact(regs, m.b), sm = div_exact(smem, m.b);
-    if (kPolicy == ROOMIE_WALK_DETAILED_EQUAL) {
-        uint32_t f = min(blocks, sp.blocks_per_sm / 2);
-        if (wb) f = min(f, div_floor(sp.threads_per_sm / 64u, wb));
-        if (rg) f = min(f, div_floor(sp.regs_per_sm / 2, rg));
-        if (sm) f = min(f, div_floor(sp.smem_per_sm / 2, sm));
-        m.fit = f;
-    } else {
-        m.wb = wb; m.rg = rg; m.sm = sm;
+__device__ __forceinline__ void fetch_ahead(CoModel& m, const uint4* __restrict__ records,
+                                            const unsigned long long* __restrict__ side) {
+    if (m.more) {
+        m.ahead = __ldg(&records[m.next_rec]);
+        m.side_ahead = __ldg(&side[m.next_side]);
+        ++m.next_rec; ++m.next_side; --m.more;
     }
+}
+
+__device__ __forceinline__ void open_model(CoModel& m, const uint4* __restrict__ records,
+                                           const unsigned long long* __restrict__ side, uint32_t first_rec,
+                                           uint32_t first_side, uint32_t n) {
+    m.rec = __ldg(&records[first_rec]);
+    m.side = __ldg(&side[first_side]);
+    m.pending = n - 1; m.more = n - 1;
+    m.next_rec = first_rec + 1; m.next_side = first_side + 1;
+    fetch_ahead(m, records, side);
+    m.idle = 0; m.began = 0; m.lost = 0.0; m.alive = true;
+    m.left = (unsigned long long)(m.rec.y - m.rec.x) * side_blocks(m.side);
 }
 
 // the active kernel is done: the next one takes its place (after the gap between them), and the one after
 // that is fetched
-template <int kPolicy>
-__device__ __forceinline__ void next_kernel(CoModel& m, const roomie_gpu_spec& sp, unsigned long long now) {
+__device__ __forceinline__ void next_kernel(CoModel& m, const uint4* __restrict__ records,
+                                            const unsigned long long* __restrict__ side, unsigned long long now) {
     if (m.pending == 0) { m.alive = false; return; }
     const uint32_t ended = m.rec.y;
-    m.rec = m.ahead;
+    m.rec = m.ahead; m.side = m.side_ahead;
     --m.pending;
-    if (m.more) { m.ahead = __ldg(m.at); ++m.at; --m.more; }
+    fetch_ahead(m, records, side);
     m.idle = m.rec.x - ended;
-    start_kernel<kPolicy>(m, sp, now);
+    m.left = (unsigned long long)(m.rec.y - m.rec.x) * side_blocks(m.side);
+    if (m.idle == 0) m.began = now;
 }
 
-template <int kPolicy>
-__device__ __forceinline__ void open_model(CoModel& m, const uint4* first, uint32_t n, const roomie_gpu_spec& sp) {
-    m.rec = __ldg(first);
-    m.pending = n - 1;
-    m.at = first + 1;
-    m.more = n - 1;
-    if (m.more) { m.ahead = __ldg(m.at); ++m.at; --m.more; }
-    m.idle = 0; m.began = 0; m.lost = 0.0; m.alive = true;
-    start_kernel<kPolicy>(m, sp, 0);
-}
-
-// blocks of `lo`'s kernel that fit beside all blocks of `hi`'s
-__device__ __forceinline__ uint32_t remainder_blocks(const CoModel& hi, const CoModel& lo, const roomie_gpu_spec& sp) {
-    const uint32_t left_w = sp.threads_per_sm / 32u - (hi.rec.z >> kWarpShift);
-    const uint32_t left_r = sp.regs_per_sm - (hi.rec.z & ((1u << kWarpShift) - 1u));
-    const uint32_t left_s = sp.smem_per_sm - (hi.rec.w & ((1u << 22) - 1u));
-    const uint32_t left_b = sp.blocks_per_sm - (hi.rec.w >> 22);
-    uint32_t f = min(lo.rec.w >> 22, left_b);
-    if (lo.wb) f = min(f, div_floor(left_w, lo.wb));
-    if (lo.rg) f = min(f, div_floor(left_r, lo.rg));
-    if (lo.sm) f = min(f, div_floor(left_s, lo.sm));
+// blocks of `lo`'s kernel that fit beside all blocks of `hi`'s (what is left of every resource)
+__device__ __forceinline__ uint32_t remainder_blocks(uint32_t hi_z, uint32_t hi_w, uint32_t lo_w, unsigned long long lo_side,
+                                                     const roomie_gpu_spec& sp) {
+    const uint32_t left_w = sp.threads_per_sm / 32u - (hi_z >> kWarpShift);
+    const uint32_t left_r = sp.regs_per_sm - (hi_z & ((1u << kWarpShift) - 1u));
+    const uint32_t left_s = sp.smem_per_sm - (hi_w & ((1u << 22) - 1u));
+    const uint32_t left_b = sp.blocks_per_sm - (hi_w >> 22);
+    const uint32_t wb = side_warps(lo_side), rb = side_regs(lo_side), sb = side_smem(lo_side);
+    uint32_t f = min(lo_w >> 22, left_b);
+    f = min(f, wb ? div_floor(left_w, wb) : f);
+    f = min(f, rb ? div_floor(left_r, rb) : f);
+    f = min(f, sb ? div_floor(left_s, sb) : f);
     return f;
-}
-
-// one model's share of an event of `step` ticks during which it ran with `bt` of its blocks (or idled)
-template <int kPolicy>
-__device__ __forceinline__ void advance(CoModel& m, uint32_t bt, unsigned long long until, unsigned long long step,
-                                        unsigned long long now, const double* s_inv, const roomie_gpu_spec& sp) {
-    if (m.idle) {
-        m.idle -= (uint32_t)step;
-        if (m.idle == 0) m.began = now;
-        return;
-    }
-    if (bt != m.b) m.lost = __fma_rn(__ull2double_rn(step * (m.b - bt)), s_inv[m.b], m.lost);
-    if (until == step) { next_kernel<kPolicy>(m, sp, now); return; }
-    m.left -= step * bt;
-    if (bt == m.b) m.full -= (uint32_t)step;
-    else m.full = (uint32_t)div_ceil(m.left, m.b, s_inv[m.b]);
 }
 
 template <int kPolicy>
@@ -248,6 +266,8 @@ __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(Detaile
     uint32_t* next_walk = g.hist + kSortBuckets + 1;
     const roomie_gpu_spec sp = g.spec;
     const PhiCap cap = g.lib.cap;
+    const uint4* __restrict__ records = g.lib.records;
+    const unsigned long long* __restrict__ side = g.side;
     const int lane = threadIdx.x & 31;
     const unsigned long long kNever = ~0ull;
 
@@ -271,8 +291,8 @@ __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(Detaile
                 if (i < n_kept) {
                     slot = g.order[i];
                     const WalkSeed s = g.seeds[slot];
-                    open_model<kPolicy>(A, g.lib.records + s.recA, s.nA, sp);
-                    open_model<kPolicy>(B, g.lib.records + s.recB, s.nB, sp);
+                    open_model(A, records, side, s.recA, s.sideA, s.nA);
+                    open_model(B, records, side, s.recB, s.sideB, s.nB);
                     now = 0; events = 0; busy = true;
                     limit = 2u * (s.nA + s.nB) + 2u;
                 } else drained = true;
@@ -281,28 +301,52 @@ __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(Detaile
         if (__all_sync(0xffffffffu, drained)) break;
         if (!busy) continue;
 
-        // one event: blocks each kernel runs with until something changes
+        // ---- one event.  Blocks each kernel runs with until something changes: all of its own unless both
+        // kernels are active and their combined demand exceeds the SM (Eq. 2) ----
         ++events;
-        uint32_t btA = A.b, btB = B.b;
-        if (A.idle == 0 && B.idle == 0 && phi_exceeds(cap.lo - A.rec.z, cap.hi - A.rec.w, B.rec.z, B.rec.w)) {
-            if (kPolicy == ROOMIE_WALK_DETAILED_EQUAL) {
-                const bool a_first = A.began <= B.began;
-                btA = A.fit; btB = B.fit;
-                if (btA == 0 && btB == 0) { if (a_first) btA = A.b; else btB = B.b; }
-                else if (btA == 0) btB = B.b;
-                else if (btB == 0) btA = A.b;
-            } else {
-                const bool a_first = kPolicy == ROOMIE_WALK_DETAILED_PRIORITY || A.began <= B.began;
-                if (a_first) btB = remainder_blocks(A, B, sp);
-                else btA = remainder_blocks(B, A, sp);
-            }
+        const uint32_t bA = side_blocks(A.side), bB = side_blocks(B.side);
+        const bool actA = A.idle == 0, actB = B.idle == 0;
+        const bool contend = actA && actB && phi_exceeds(cap.lo - A.rec.z, cap.hi - A.rec.w, B.rec.z, B.rec.w);
+        const bool a_first = kPolicy == ROOMIE_WALK_DETAILED_PRIORITY || A.began <= B.began;
+        uint32_t btA, btB;
+        if (kPolicy == ROOMIE_WALK_DETAILED_EQUAL) {
+            const uint32_t fA = side_half_fit(A.side), fB = side_half_fit(B.side);
+            const bool none = fA == 0 && fB == 0;
+            btA = fB == 0 ? (none && !a_first ? 0u : bA) : fA;      // the other does not fit: all my blocks
+            btB = fA == 0 ? (none && a_first ? 0u : bB) : fB;
+        } else {
+            const uint32_t rest = remainder_blocks(a_first ? A.rec.z : B.rec.z, a_first ? A.rec.w : B.rec.w,
+                                                   a_first ? B.rec.w : A.rec.w, a_first ? B.side : A.side, sp);
+            btA = a_first ? bA : rest;
+            btB = a_first ? rest : bB;
         }
-        const unsigned long long untilA = A.idle ? A.idle : btA == A.b ? A.full : btA ? div_ceil(A.left, btA, s_inv[btA]) : kNever;
-        const unsigned long long untilB = B.idle ? B.idle : btB == B.b ? B.full : btB ? div_ceil(B.left, btB, s_inv[btB]) : kNever;
+        btA = contend ? btA : bA;
+        btB = contend ? btB : bB;
+        // ticks to the next event: a gap ends, or a kernel has done its block-ticks at btX per tick
+        const unsigned long long runA = div_ceil(A.left, btA ? btA : 1u, s_inv[btA ? btA : 1u]);
+        const unsigned long long runB = div_ceil(B.left, btB ? btB : 1u, s_inv[btB ? btB : 1u]);
+        const unsigned long long untilA = actA ? (btA ? runA : kNever) : A.idle;
+        const unsigned long long untilB = actB ? (btB ? runB : kNever) : B.idle;
         const unsigned long long step = untilA < untilB ? untilA : untilB;
         now += step;
-        advance<kPolicy>(A, btA, untilA, step, now, s_inv, sp);
-        advance<kPolicy>(B, btB, untilB, step, now, s_inv, sp);
+        // model A
+        {
+            const bool done = actA && untilA == step;
+            if (actA && btA != bA) A.lost = __fma_rn(__ull2double_rn(step * (bA - btA)), s_inv[bA], A.lost);
+            if (!actA && A.idle == (uint32_t)step) A.began = now;
+            A.idle = actA ? 0u : A.idle - (uint32_t)step;
+            A.left -= (actA && !done) ? step * btA : 0ull;
+            if (done) next_kernel(A, records, side, now);
+        }
+        // model B
+        {
+            const bool done = actB && untilB == step;
+            if (actB && btB != bB) B.lost = __fma_rn(__ull2double_rn(step * (bB - btB)), s_inv[bB], B.lost);
+            if (!actB && B.idle == (uint32_t)step) B.began = now;
+            B.idle = actB ? 0u : B.idle - (uint32_t)step;
+            B.left -= (actB && !done) ? step * btB : 0ull;
+            if (done) next_kernel(B, records, side, now);
+        }
         if (events >= limit && A.alive && B.alive) {
             atomicOr(g.status, ROOMIE_FLAG_WORKSPACE);
             A.alive = false;

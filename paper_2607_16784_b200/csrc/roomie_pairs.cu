@@ -602,7 +602,7 @@ static void pair_of_host(uint64_t p, uint32_t P, uint32_t& a, uint32_t& b) {
 
 static uint32_t host_grid_count(uint32_t q, uint32_t A) { return (A == 0 || A > q) ? q : A; }
 
-struct Need { uint64_t walks, tiles; };
+struct Need { uint64_t walks, tiles, side; };     // side: 8-byte per-kernel records of the Section 3.2 simulator
 constexpr uint64_t kDetailedExtraTiles = 160;     // 5 KB: the 1026-word bucket table of the walk sort
 
 // upper bound of walk slots and tiles for pairs [p0, p1): a walk of a pair has at most
@@ -657,6 +657,7 @@ static bool batch_need(const roomie_library* lib, const roomie_opts* o, bool exp
     need.walks = (explicit_pair ? 1 : (p1 - p0)) * (uint64_t)slots;
     if (detailed) tiles = need.walks + kDetailedExtraTiles;       // one result per walk slot + the sort's bucket table
     need.tiles = tiles;
+    need.side = !detailed ? 0 : explicit_pair ? (uint64_t)(off[ea + 1] - off[ea]) + (off[eb + 1] - off[eb]) : lib->num_kernels;
     return true;
 }
 
@@ -664,7 +665,7 @@ static size_t align_up(size_t x) { return (x + 255) & ~(size_t)255; }
 
 static size_t bytes_for(const Need& n) {
     return 256 + align_up(n.walks * sizeof(WalkInfo)) + align_up(n.tiles * sizeof(TileDesc)) +
-           align_up(n.tiles * sizeof(TilePartial));
+           align_up(n.tiles * sizeof(TilePartial)) + align_up(n.side * sizeof(uint64_t));
 }
 
 static int slots_for(const roomie_library* lib, const roomie_opts* o, bool explicit_pair, uint32_t ea, uint32_t eb,
@@ -743,8 +744,8 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
     if (o->walk_mode >= ROOMIE_WALK_DETAILED_EQUAL) {
         // Section 3.2 simulator: the walks are sorted by expected length (plan, scan, scatter), then persistent
         // lanes pull them; every walk writes its result where the tile partials go.  The sort's scratch lives in
-        // the tile-descriptor area: 32 bytes per walk plus kDetailedExtraTiles descriptors are reserved, 22 bytes
-        // per walk and the bucket table are used.
+        // the tile-descriptor area: 32 bytes per walk plus kDetailedExtraTiles descriptors are reserved, 30 bytes
+        // per walk and the bucket table are used.  The per-kernel side records follow the partial results.
         unsigned char* area = reinterpret_cast<unsigned char*>(tiles);
         DetailedArgs da;
         da.lib = lv; da.ps = ps; da.slots = slots; da.n_align = o->n_align; da.start_filter = o->start_filter;
@@ -752,7 +753,20 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
         da.seeds = reinterpret_cast<WalkSeed*>(area);
         da.order = reinterpret_cast<uint32_t*>(area + need.walks * sizeof(WalkSeed));
         da.bucket = reinterpret_cast<uint16_t*>(area + need.walks * (sizeof(WalkSeed) + sizeof(uint32_t)));
-        da.hist = reinterpret_cast<uint32_t*>(area + ((need.walks * 22 + 15) & ~(uint64_t)15));
+        da.hist = reinterpret_cast<uint32_t*>(area + ((need.walks * 30 + 15) & ~(uint64_t)15));
+        da.side = reinterpret_cast<unsigned long long*>(reinterpret_cast<unsigned char*>(partials) +
+                                                        align_up(need.tiles * sizeof(TilePartial)));
+        if (ps.explicit_pair) {
+            const uint32_t* off = lib->offsets_host;
+            da.n_ranges = 2;
+            da.range[0].first_record = off[ps.a]; da.range[0].count = off[ps.a + 1] - off[ps.a]; da.range[0].first_side = 0;
+            da.range[1].first_record = off[ps.b]; da.range[1].count = off[ps.b + 1] - off[ps.b];
+            da.range[1].first_side = da.range[0].count;
+        } else {
+            da.n_ranges = 1;
+            da.range[0].first_record = 0; da.range[0].count = lib->num_kernels; da.range[0].first_side = 0;
+            da.range[1] = da.range[0];
+        }
         uint32_t qmax = 1;
         if (ps.explicit_pair) {
             const uint32_t* off = lib->offsets_host;
@@ -765,6 +779,10 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
         da.shift = 0;
         while (((2ull * qmax) >> da.shift) >= (uint64_t)kSortBuckets) ++da.shift;
         ROOMIE_CUDA_OK(cudaMemsetAsync(da.hist, 0, (kSortBuckets + 2) * sizeof(uint32_t), st));
+        uint64_t sblocks = (need.side + 255) / 256;
+        if (sblocks > (uint64_t)sm_count() * 8) sblocks = (uint64_t)sm_count() * 8;
+        detailed_side_kernel<<<(unsigned)(sblocks ? sblocks : 1), 256, 0, st>>>(da);
+        note_launch();
         uint64_t pblocks = (need.walks + 255) / 256;
         if (pblocks > (uint64_t)sm_count() * 8) pblocks = (uint64_t)sm_count() * 8;
         detailed_plan_kernel<<<(unsigned)pblocks, 256, 0, st>>>(da);
