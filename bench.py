@@ -77,8 +77,9 @@ def parse_args():
                     help="the timed region (exactly --steps steps) is run this many times; the median is reported")
     ap.add_argument("--impl", default="roomie", choices=["roomie", "reference"])
     ap.add_argument("--config", type=int, default=3, help="library configuration (0-4)")
-    ap.add_argument("--setting", default="base", choices=["base", "greedy", "lockstep_full", "detailed"],
-                    help="base: alignment (0,0); greedy: 8x8 alignments, start filter, median; lockstep_full: "
+    ap.add_argument("--setting", default="base", choices=["base", "greedy", "lockstep", "lockstep_full", "detailed"],
+                    help="base: alignment (0,0); greedy: 8x8 alignments, start filter, median; lockstep: Algorithm 1's "
+                         "lock-step walk on the 8x8 alignment grid; lockstep_full: "
                          "Algorithm 1 as printed over the full Cartesian alignment set; detailed: Section 3.2 simulator")
     ap.add_argument("--arrivals", type=int, default=10000)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -96,6 +97,8 @@ def parse_args():
 def setting_kw(name):
     if name == "lockstep_full":
         return dict(mode=1, n_align=0, start_filter=1)
+    if name == "lockstep":
+        return dict(mode=1, n_align=8, start_filter=1)
     if name == "detailed":                              # Section 3.2 simulator, equal partition, alignment (0, 0)
         return dict(mode=2, n_align=1, start_filter=0)
     return dict(mode=0, n_align=1, start_filter=0) if name == "base" else dict(mode=0, n_align=8, start_filter=1)
@@ -106,7 +109,7 @@ def oracle_sample_pairs(setting, lib):
     list where it is smaller, as on the default workload at the base setting)."""
     P = lib.num_profiles
     total = P * (P + 1) // 2
-    per_pair = 2.0 * float(lib.q().mean()) * {"base": 1.0, "detailed": 1.6, "greedy": 26.0}.get(setting, 0.0)
+    per_pair = 2.0 * float(lib.q().mean()) * {"base": 1.0, "detailed": 1.6, "greedy": 26.0, "lockstep": 13.0}.get(setting, 0.0)
     if setting == "lockstep_full":
         per_pair = float(lib.q().mean()) ** 2 * float(lib.q().mean()) / 3.0          # one walk per alignment
     return int(max(1, min(total, 1.0e9 / max(per_pair, 1.0))))
@@ -414,6 +417,12 @@ def main():
                         "unit": "G cell visits/s", "frac": (ach / peak_visits) if ach else None,
                         "peak_source": "derived: 148 SMs x 128 lanes x SM clock / 53 lane-instructions per visit",
                         "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix, "traffic": None}
+        elif args.setting == "lockstep":
+            roofline = {"bound": "hbm", "kernel": "lockstep_tiles_kernel", "achieved": 32.0 * evals_rank / kernel_s / 1e9 / launches_per_matrix if walk_launches else None,
+                        "peak": peak, "unit": "GB/s", "frac": (32.0 * evals_rank / kernel_s / 1e9 / launches_per_matrix / peak) if walk_launches else None,
+                        "peak_source": peak_src, "algorithmic_bytes_per_launch": 32.0 * evals_rank / launches_per_matrix,
+                        "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix, "traffic": None,
+                        "note": "32 B per pairing (two 16-byte records), served from L2 when the library fits there"}
         elif args.setting == "detailed":
             roofline = {"bound": "alu", "kernel": "detailed_walk_kernel", "achieved": evals_rank / kernel_s / 1e9 if walk_launches else None,
                         "peak": None, "unit": "G events/s", "frac": None,

@@ -31,6 +31,7 @@
 
 constexpr int kSortBuckets = 1024;
 constexpr int kDetailedThreads = 128;
+constexpr int kEventsPerLook = 4;          // events a lane simulates between two looks at the walk queue
 
 struct WalkSeed {              // what a lane needs to start a walk, written by the plan kernel
     uint32_t recA, recB;       // global index of each model's first record of the alignment
@@ -75,15 +76,12 @@ __device__ __forceinline__ uint32_t div_floor(uint32_t x, uint32_t d) {
     q += (r >= 0 && (uint32_t)r >= d) ? 1u : 0u;
     return q;
 }
-// ceil(x / d) for x < 2^45, 1 <= d <= 255, with inv = the double nearest to 1/d: the product is within 2^-7 of
-// the quotient, so its integer part is at most one off
-__device__ __forceinline__ unsigned long long div_ceil(unsigned long long x, uint32_t d, double inv) {
-    long long q = __double2ll_rz(__dmul_rn(__ull2double_rn(x), inv));
-    long long r = (long long)x - q * (long long)d;
-    const bool low = r < 0, high = r >= (long long)d;
-    q += high ? 1 : (low ? -1 : 0);
-    r += low ? (long long)d : (high ? -(long long)d : 0);
-    return (unsigned long long)q + (r != 0 ? 1ull : 0ull);
+// ceil(x / d) for x < 2^47, 1 <= d <= 255, with magic = ceil(2^64 / d) (2^64 - 1 for d = 1): the high half of
+// y * magic is floor(y / d) exactly for every y < 2^56 (the excess of magic over 2^64 / d is below 1, so the error
+// of the product is below y, far less than the 2^64 / d that separates a quotient from the next integer)
+__device__ __forceinline__ unsigned long long div_ceil(unsigned long long x, uint32_t d, unsigned long long magic) {
+    const unsigned long long y = x + d - 1;
+    return d == 1 ? x : __umul64hi(y, magic);
 }
 
 __device__ __forceinline__ uint32_t side_blocks(unsigned long long s) { return (uint32_t)s & 255u; }
@@ -259,8 +257,12 @@ __device__ __forceinline__ uint32_t remainder_blocks(uint32_t hi_z, uint32_t hi_
 
 template <int kPolicy>
 __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(DetailedArgs g) {
-    __shared__ double s_inv[256];
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_inv[i] = i ? __ddiv_rn(1.0, (double)i) : 0.0;
+    __shared__ double s_inv[256];                    // 1 / b: a tick with b~ of b blocks loses (b - b~) / b
+    __shared__ unsigned long long s_magic[256];      // ceil(2^64 / d): division by a block count
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) {
+        s_inv[i] = i ? __ddiv_rn(1.0, (double)i) : 0.0;
+        s_magic[i] = i > 1 ? 0xffffffffffffffffull / (unsigned long long)i + 1ull : 0xffffffffffffffffull;
+    }
     __syncthreads();
     const uint32_t n_kept = g.hist[kSortBuckets];
     uint32_t* next_walk = g.hist + kSortBuckets + 1;
@@ -299,8 +301,11 @@ __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(Detaile
             }
         }
         if (__all_sync(0xffffffffu, drained)) break;
-        if (!busy) continue;
 
+        // a few events between two looks at the queue (a lane that finishes in between idles for the rest)
+#pragma unroll 1
+        for (int rep = 0; rep < kEventsPerLook; ++rep) {
+        if (!busy) continue;
         // ---- one event.  Blocks each kernel runs with until something changes: all of its own unless both
         // kernels are active and their combined demand exceeds the SM (Eq. 2) ----
         ++events;
@@ -323,8 +328,8 @@ __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(Detaile
         btA = contend ? btA : bA;
         btB = contend ? btB : bB;
         // ticks to the next event: a gap ends, or a kernel has done its block-ticks at btX per tick
-        const unsigned long long runA = div_ceil(A.left, btA ? btA : 1u, s_inv[btA ? btA : 1u]);
-        const unsigned long long runB = div_ceil(B.left, btB ? btB : 1u, s_inv[btB ? btB : 1u]);
+        const unsigned long long runA = div_ceil(A.left, btA ? btA : 1u, s_magic[btA ? btA : 1u]);
+        const unsigned long long runB = div_ceil(B.left, btB ? btB : 1u, s_magic[btB ? btB : 1u]);
         const unsigned long long untilA = actA ? (btA ? runA : kNever) : A.idle;
         const unsigned long long untilB = actB ? (btB ? runB : kNever) : B.idle;
         const unsigned long long step = untilA < untilB ? untilA : untilB;
@@ -359,6 +364,7 @@ __global__ void __launch_bounds__(kDetailedThreads) detailed_walk_kernel(Detaile
             out.di = (float)A.lost; out.dj = (float)B.lost; out.V = 0; out.ties = 0; out.pad = 0;
             g.partials[slot] = out;
             busy = false;
+        }
         }
     }
 }
