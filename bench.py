@@ -44,8 +44,8 @@ UNIT = "evals/s"
 # dram__bytes_read.sum + dram__bytes_write.sum on the default workload (configuration 3, 512 profiles, base)
 MEASURED_WALK_TRAFFIC = {(3, 512, "base"): 38328832 + 62720}
 # smsp__inst_executed.sum x 32 lanes / scored pairings: lane-instructions the kernel spends per evaluation
-# (128-profile case of configuration 3)
-WALK_LANE_INSTR_PER_EVAL = {"base": 80.0, "greedy": 80.0}
+# (128-profile case of configuration 3; the greedy setting's short walks from late start indices cost a little more)
+WALK_LANE_INSTR_PER_EVAL = {"base": 80.0, "greedy": 86.4}
 SM_COUNT, LANES_PER_SM = 148, 128
 
 
@@ -82,6 +82,8 @@ def parse_args():
                          "lock-step walk on the 8x8 alignment grid; lockstep_full: "
                          "Algorithm 1 as printed over the full Cartesian alignment set; detailed: Section 3.2 simulator")
     ap.add_argument("--arrivals", type=int, default=10000)
+    ap.add_argument("--cluster-gpus", type=int, default=None, help="modelled GPUs of the placement cluster (default: the configuration's 64 or 8)")
+    ap.add_argument("--cluster-slots", type=int, default=None, help="resident slots per modelled GPU (more than 8 takes the generic placement kernel)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--profiles", type=int, default=None,
                     help="number of profiles drawn from the configuration's recipe (fewer: ncu captures; 4096 on "
@@ -115,12 +117,13 @@ def oracle_sample_pairs(setting, lib):
     return int(max(1, min(total, 1.0e9 / max(per_pair, 1.0))))
 
 
-def make_inputs(cfg, num_profiles, arrivals, rank=0):
+def make_inputs(cfg, num_profiles, arrivals, rank=0, gpus=None, slots=None):
     seed = rs.config_seed(cfg)
     lib = rs.make_library(cfg, seed=seed, num_profiles=num_profiles)
     ccfg = cfg if rs.CONFIGS[cfg].num_gpus else 2          # cluster shape of the online-placement config
     # placement is replicated, not sharded: every rank places its own arrival stream over the common library
-    cl = rs.make_cluster(ccfg, seed=seed + 7919 * rank, num_profiles=lib.num_profiles, num_arrivals=arrivals)
+    cl = rs.make_cluster(ccfg, seed=seed + 7919 * rank, num_profiles=lib.num_profiles, num_arrivals=arrivals,
+                         num_gpus=gpus, max_residents=slots)
     return lib, cl
 
 
@@ -201,7 +204,7 @@ def run_reference(args, rank, world):
         return
     import oracle
     oracle.build()
-    lib, cl = make_inputs(args.config, args.profiles, args.arrivals)
+    lib, cl = make_inputs(args.config, args.profiles, args.arrivals, 0, args.cluster_gpus, args.cluster_slots)
     kw = setting_kw(args.setting)
     P = lib.num_profiles
     total_pairs = P * (P + 1) // 2
@@ -246,7 +249,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    lib, cl = make_inputs(args.config, args.profiles, args.arrivals, rank)
+    lib, cl = make_inputs(args.config, args.profiles, args.arrivals, rank, args.cluster_gpus, args.cluster_slots)
     kw = setting_kw(args.setting)
     P, K = lib.num_profiles, lib.num_kernels
     G, R = cl.num_gpus, cl.max_residents

@@ -633,6 +633,8 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
     if (tid == 0) *g.tick = tick0 + g.n;
 }
 
+#include "roomie_place_slots.cuh"
+
 }  // namespace roomie
 
 using namespace roomie;
@@ -670,6 +672,20 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
     a.arr_id = arr_id; a.arr_life = arr_life; a.n = n; a.lambda = opts->lambda;
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (num_streams == 1 && a.R <= (uint32_t)kSlotLanes && a.G <= (1024u - 32u) / kSlotLanes) {
+        // one stream, up to 8 slots per GPU: one lane per resident slot (the shortest dependent chain; a batch of
+        // independent streams is a throughput problem and takes the one-lane-per-GPU kernel below instead)
+        a.matrix_mode = 1; a.pair_cache = 1; a.gpus_per_warp = 32 / kSlotLanes; a.chunk = kSlotChunk;
+        const uint32_t threads = ((a.G * kSlotLanes + 31) / 32) * 32 + 32;   // one more warp that owns no GPU
+        const size_t bytes = (size_t)slot_layout(threads, a.G).total * sizeof(float);
+        auto kern = (a.admit_rule == 0 && a.objective == 0) ? place_slots_kernel<true> : place_slots_kernel<false>;
+        if (bytes > 48 * 1024)
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+        kern<<<1, threads, bytes, st>>>(a);
+        note_launch();
+        ROOMIE_CUDA_OK(cudaGetLastError());
+        return ROOMIE_OK;
+    }
     const size_t GR = (size_t)a.G * a.R;
     // many independent streams: a short staging chunk keeps the CTA small enough (44.4 KB) for 5 per SM
     a.chunk = num_streams > 1 ? 32u : kArrChunk;
