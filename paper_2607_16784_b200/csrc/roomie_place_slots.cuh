@@ -1,4 +1,4 @@
-// Algorithm 2 with ONE LANE PER RESIDENT SLOT: clusters of up to 8 slots per modelled GPU and up to 128 GPUs.
+// Algorithm 2 with ONE LANE PER RESIDENT SLOT: clusters of up to 8 slots per modelled GPU and up to 124 GPUs.
 // Included by roomie_place.cu inside namespace roomie.
 //
 // The arrival stream is a dependent chain: what bounds it is the number of instructions one warp executes per
