@@ -374,6 +374,51 @@ def test_placement_edge_cases(rm, oracle):
     assert np.array_equal(gpu, want.gpu)
 
 
+@pytest.mark.parametrize("shape", [(120, 8), (124, 8), (125, 8), (17, 7), (3, 5), (1, 8), (64, 1)])
+def test_placement_cluster_shapes_around_the_kernel_limits(rm, oracle, shape):
+    """Shapes on both sides of the limits that select a placement kernel (one lane per resident slot up to 124 GPUs
+    of at most 8 slots, one lane per GPU beyond), slot counts that leave lanes of a group unused, GPU counts that
+    leave groups of a warp unused: every decision, the final state and the means against the oracle."""
+    G, R = shape
+    rng = np.random.default_rng(100 * G + R)
+    P, n = 48, 1500
+    Pm = (rng.random((P, P)) * 0.35).astype(np.float32)
+    aid = rng.integers(0, P, n).astype(np.int32)
+    life = rng.geometric(1.0 / (2.0 * G), n).astype(np.uint32)          # about two residents per GPU in steady state
+    ids = np.full(G * R, -1, np.int32); exp = np.zeros(G * R, np.uint32); cnt = np.zeros(G, np.uint32)
+    for g in range(0, G, 3):                                             # some GPUs start with residents
+        k = min(R, 1 + g % 3)
+        ids[g * R:g * R + k] = rng.integers(0, P, k); exp[g * R:g * R + k] = rng.integers(5, 60, k); cnt[g] = k
+    for lam in (0.5, 1e9):
+        st = rm.ClusterState(G, R, ids, exp, cnt, 3)
+        gpu, mean, mu_arr = rm.place(Pm, st, aid, life, lam)
+        want = oracle.place(Pm, G, R, ids, exp, cnt, 3, aid, life, lam)
+        assert np.array_equal(gpu.cpu().numpy(), want.gpu)
+        assert np.array_equal(mean.cpu().numpy().view(np.uint32), want.mean.view(np.uint32))
+        assert np.array_equal(mu_arr.cpu().numpy().view(np.uint32), want.mu_arr.view(np.uint32))
+        assert np.array_equal(st.ids.cpu().numpy(), want.ids) and np.array_equal(to_np_u32(st.expiry), want.expiry)
+        assert np.array_equal(to_np_u32(st.count), want.count) and int(st.tick.item()) == want.tick
+
+
+def test_placement_short_lifetimes_reuse_slots_at_once(rm, oracle):
+    """Lifetimes of one to four arrivals on a tiny cluster with everything admitted: a slot is freed and taken again
+    within the distance the kernels fetch ahead, the same GPU wins several arrivals in a row, residents leave while
+    the terms fetched for them are still in flight - the cases the recent-arrival terms exist for."""
+    rng = np.random.default_rng(77)
+    P, n = 40, 4000
+    Pm = (rng.random((P, P)) * 0.3).astype(np.float32)
+    aid = rng.integers(0, P, n).astype(np.int32)
+    for G, R, hi in ((2, 8, 5), (3, 3, 3), (1, 8, 9), (8, 4, 12), (70, 8, 200)):
+        life = rng.integers(1, hi, n).astype(np.uint32)
+        life[rng.random(n) < 0.02] = 0                                   # a few that never leave
+        st = rm.ClusterState(G, R, [-1] * (G * R), [0] * (G * R), [0] * G, 0)
+        gpu, mean, _ = rm.place(Pm, st, aid, life, 1e9)
+        want = oracle.place(Pm, G, R, [-1] * (G * R), [0] * (G * R), [0] * G, 0, aid, life, 1e9)
+        assert np.array_equal(gpu.cpu().numpy(), want.gpu), (G, R)
+        assert np.array_equal(mean.cpu().numpy().view(np.uint32), want.mean.view(np.uint32)), (G, R)
+        assert np.array_equal(st.ids.cpu().numpy(), want.ids) and np.array_equal(to_np_u32(st.expiry), want.expiry)
+
+
 def test_placement_rejects_ids_outside_the_matrix(rm, oracle):
     """Profile ids live on the device, so they are checked there: an arrival with an id outside [0, P) is not placed
     (gpu_out = -2) and changes nothing - the other decisions equal those of the stream without it; a cluster state that
