@@ -9,8 +9,10 @@
 // neighbouring diagonals from their far ends and the values go
 // straight into the histogram of an exact radix select (3 digit passes of 11/11/10 bits over the
 // float bits, which order like the non-negative values - the first one also counts the kept
-// alignments - plus, for an even count, a pass for the upper middle value).  Every pass recomputes the suffix sums; a suffix sum is accumulated in double
-// and ranked as float.
+// alignments).  For an even count the upper middle value comes out of the last digit pass as well: it is the same
+// value, the next occupied bin of the last histogram, or - when the lower middle is the largest value under its
+// 22-bit prefix - the smallest value above that prefix, which the pass tracks on the side.  Every pass recomputes the
+// suffix sums; a suffix sum is accumulated in double and ranked as float.
 //
 // One CTA per pair; both directions (delta_i, delta_j) are selected in the same passes.
 
@@ -25,16 +27,18 @@ struct FullArgs {
     uint32_t n_inv;
     float* P_out;
     unsigned long long* evals_out;
+    unsigned long long max_cells;  // upper bound of q_a * q_b over the pairs of the call (sets the size classes)
 };
 
-enum FullPass : int { kPassDigit0 = 0, kPassDigit1 = 1, kPassDigit2 = 2, kPassUpper = 3 };
+constexpr int kFullClasses = 4;   // size classes of the launch order, largest tables first
+
+enum FullPass : int { kPassDigit0 = 0, kPassDigit1 = 1, kPassDigit2 = 2 };
 
 struct FullSelect {               // state of the radix select of one direction
     uint32_t prefix;              // bits fixed so far
     uint32_t rank;                // rank still to find among the values that share the prefix
-    uint32_t value_bits;          // after digit 2: the element of rank k1
-    uint32_t count_le;            // pass kPassUpper: values <= value
-    uint32_t min_gt;              // pass kPassUpper: smallest value bits above value
+    uint32_t value_bits;          // after digit 2: the element of rank k1 (the lower middle)
+    uint32_t upper_bits;          // after digit 2: the element of rank k1 + 1, if the count is even
 };
 
 // walks every diagonal of the pair once; `visit(vi_bits, vj_bits, walk_len)` is called for every
@@ -107,8 +111,10 @@ __device__ __forceinline__ void full_walk(const uint4* __restrict__ A, const uin
 
 // finds the bin that holds the element of rank `rank` in hist[0..kFullBins); every thread gets the
 // bin and the rank inside it.  s_scan: kFullThreads/32 + 2 words of shared scratch.
+// With `next_bin` the caller also learns whether the element of rank + 1 is in the same bin (next_bin = bin) or which
+// is the next occupied bin (kFullBins when there is none).
 __device__ __forceinline__ void full_locate(const uint32_t* hist, uint32_t rank, uint32_t* s_scan, uint32_t& bin,
-                                            uint32_t& rank_in_bin) {
+                                            uint32_t& rank_in_bin, uint32_t* next_bin = nullptr) {
     constexpr int kPer = kFullBins / kFullThreads;                 // bins per thread
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     uint32_t h[kPer], mine = 0;
@@ -135,29 +141,57 @@ __device__ __forceinline__ void full_locate(const uint32_t* hist, uint32_t rank,
     bin = s_scan[kFullThreads / 32];
     rank_in_bin = s_scan[kFullThreads / 32 + 1];
     __syncthreads();
+    if (next_bin) {
+        if (rank_in_bin + 1 < hist[bin]) *next_bin = bin;
+        else {
+            // lowest occupied bin above `bin`: every thread proposes the first of its own bins, the minimum wins
+            if (threadIdx.x == 0) s_scan[kFullThreads / 32] = kFullBins;
+            __syncthreads();
+            uint32_t cand = kFullBins;
+#pragma unroll
+            for (int k = kPer - 1; k >= 0; --k) {
+                const uint32_t b = threadIdx.x * kPer + k;
+                if (b > bin && h[k]) cand = b;
+            }
+            if (cand < (uint32_t)kFullBins) atomicMin(&s_scan[kFullThreads / 32], cand);
+            __syncthreads();
+            *next_bin = s_scan[kFullThreads / 32];
+            __syncthreads();
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kFullThreads) lockstep_full_kernel(FullArgs g) {
     __shared__ uint32_t s_hist[2][kFullBins];
     __shared__ uint32_t s_scan[kFullThreads / 32 + 2];
-    __shared__ uint32_t s_red[4];                    // count_le_i, count_le_j, min_gt_i, min_gt_j
+    __shared__ uint32_t s_gt[2];                     // per direction: smallest value above the 22-bit prefix
     __shared__ unsigned long long s_ev;
     __shared__ uint32_t s_n;
     extern __shared__ float s_inv[];
 
-    for (uint32_t i = threadIdx.x; i < g.n_inv; i += kFullThreads) s_inv[i] = __ldg(&g.inv_table[i]);
-    for (uint32_t local = blockIdx.x; local < g.ps.n_pairs; local += gridDim.x) {
+    // The grid is kFullClasses x n_pairs CTAs: CTA c * n_pairs + p takes pair p if the pair's table falls into size
+    // class c (class 0: at least a quarter of the largest possible table, then a factor of four per class) and
+    // leaves at once otherwise, so that the largest tables start first and the small ones fill the tail.
+    {
+        const uint32_t local = blockIdx.x % g.ps.n_pairs, cls = blockIdx.x / g.ps.n_pairs;
         uint32_t a, b;
         pair_of(g.ps, g.lib.P, local, a, b);
         const uint32_t offa = g.lib.offsets[a], offb = g.lib.offsets[b];
         const uint32_t na = g.lib.offsets[a + 1] - offa, nb = g.lib.offsets[b + 1] - offb;
+        const unsigned long long cells = (unsigned long long)na * nb;
+        uint32_t mine = kFullClasses - 1;
+#pragma unroll
+        for (int c = kFullClasses - 2; c >= 0; --c)
+            if (cells >= (g.max_cells >> (2 * c + 2))) mine = c;
+        if (mine != cls) return;
+        for (uint32_t i = threadIdx.x; i < g.n_inv; i += kFullThreads) s_inv[i] = __ldg(&g.inv_table[i]);
         const uint4* A = g.lib.records + offa;
         const uint4* B = g.lib.records + offb;
         FullSelect sel[2] = {};
         uint32_t n = 0;
-        for (int pass = kPassDigit0; pass <= kPassUpper; ++pass) {
+        for (int pass = kPassDigit0; pass <= kPassDigit2; ++pass) {
             for (uint32_t i = threadIdx.x; i < 2 * kFullBins; i += kFullThreads) (&s_hist[0][0])[i] = 0;
-            if (threadIdx.x == 0) { s_ev = 0; s_n = 0; s_red[0] = s_red[1] = 0; s_red[2] = s_red[3] = 0xffffffffu; }
+            if (threadIdx.x == 0) { s_ev = 0; s_n = 0; s_gt[0] = s_gt[1] = 0xffffffffu; }
             __syncthreads();
             if (pass == kPassDigit0) {                                   // first digit, count and walk lengths
                 uint32_t cnt = 0;
@@ -169,24 +203,24 @@ __global__ void __launch_bounds__(kFullThreads) lockstep_full_kernel(FullArgs g)
                 });
                 atomicAdd(&s_n, cnt);
                 atomicAdd(&s_ev, ev);
-            } else if (pass <= kPassDigit2) {
-                const int shift = pass == kPassDigit1 ? 10 : 0;
-                const uint32_t mask = pass == kPassDigit2 ? 1023u : 2047u;
-                const int pshift = pass == kPassDigit1 ? 21 : 10;        // bits already fixed: v >> pshift
+            } else if (pass == kPassDigit1) {
                 const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
                 full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
-                    if ((vi >> pshift) == pi) atomicAdd(&s_hist[0][(vi >> shift) & mask], 1u);
-                    if ((vj >> pshift) == pj) atomicAdd(&s_hist[1][(vj >> shift) & mask], 1u);
+                    if ((vi >> 21) == pi) atomicAdd(&s_hist[0][(vi >> 10) & 2047u], 1u);
+                    if ((vj >> 21) == pj) atomicAdd(&s_hist[1][(vj >> 10) & 2047u], 1u);
                 });
             } else {
-                const uint32_t ti = sel[0].value_bits, tj = sel[1].value_bits;
-                uint32_t le_i = 0, le_j = 0, gt_i = 0xffffffffu, gt_j = 0xffffffffu;
+                // last digit; on the side, the smallest value whose upper 22 bits lie above the prefix (the upper
+                // middle of an even count when the lower middle is the largest value under the prefix)
+                const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
+                uint32_t gt_i = 0xffffffffu, gt_j = 0xffffffffu;
                 full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
-                    if (vi <= ti) ++le_i; else gt_i = min(gt_i, vi);
-                    if (vj <= tj) ++le_j; else gt_j = min(gt_j, vj);
+                    const uint32_t ui = vi >> 10, uj = vj >> 10;
+                    if (ui == pi) atomicAdd(&s_hist[0][vi & 1023u], 1u); else if (ui > pi) gt_i = min(gt_i, vi);
+                    if (uj == pj) atomicAdd(&s_hist[1][vj & 1023u], 1u); else if (uj > pj) gt_j = min(gt_j, vj);
                 });
-                atomicAdd(&s_red[0], le_i); atomicAdd(&s_red[1], le_j);
-                atomicMin(&s_red[2], gt_i); atomicMin(&s_red[3], gt_j);
+                if (gt_i != 0xffffffffu) atomicMin(&s_gt[0], gt_i);
+                if (gt_j != 0xffffffffu) atomicMin(&s_gt[1], gt_j);
             }
             __syncthreads();
             if (pass == kPassDigit0) {
@@ -195,32 +229,26 @@ __global__ void __launch_bounds__(kFullThreads) lockstep_full_kernel(FullArgs g)
                 if (n == 0) break;
                 sel[0].rank = sel[1].rank = (n - 1) / 2;
             }
-            if (pass <= kPassDigit2) {
-                const int bits = pass == kPassDigit2 ? 10 : 11;
-                for (int dir = 0; dir < 2; ++dir) {
-                    uint32_t bin, r;
-                    full_locate(s_hist[dir], sel[dir].rank, s_scan, bin, r);
-                    sel[dir].prefix = (sel[dir].prefix << bits) | bin;
-                    sel[dir].rank = r;
-                }
+            const int bits = pass == kPassDigit2 ? 10 : 11;
+            for (int dir = 0; dir < 2; ++dir) {
+                uint32_t bin, r, next = 0;
+                full_locate(s_hist[dir], sel[dir].rank, s_scan, bin, r, pass == kPassDigit2 ? &next : nullptr);
+                const uint32_t group = sel[dir].prefix;                  // the bits fixed before this pass
+                sel[dir].prefix = (group << bits) | bin;
+                sel[dir].rank = r;
                 if (pass == kPassDigit2) {
-                    sel[0].value_bits = sel[0].prefix; sel[1].value_bits = sel[1].prefix;
-                    sel[0].count_le = sel[1].count_le = n;               // odd count: both middles are this element
-                    if (n & 1u) break;
+                    sel[dir].value_bits = sel[dir].prefix;
+                    sel[dir].upper_bits = next < (uint32_t)kFullBins ? ((group << 10) | next) : s_gt[dir];
                 }
-            } else {
-                sel[0].count_le = s_red[0]; sel[1].count_le = s_red[1];
-                sel[0].min_gt = s_red[2]; sel[1].min_gt = s_red[3];
             }
             __syncthreads();
         }
         if (threadIdx.x == 0) {
             float med[2] = {0.0f, 0.0f};
             if (n > 0) {
-                const uint32_t k2 = n / 2;                         // upper middle (equals the lower one for odd n)
                 for (int dir = 0; dir < 2; ++dir) {
                     const float lo = __uint_as_float(sel[dir].value_bits);
-                    const float hi = k2 < sel[dir].count_le ? lo : __uint_as_float(sel[dir].min_gt);
+                    const float hi = (n & 1u) ? lo : __uint_as_float(sel[dir].upper_bits);   // odd count: one middle
                     med[dir] = 0.5f * (lo + hi);
                 }
             }

@@ -705,8 +705,17 @@ static int run_lockstep_full(const roomie_library* lib, const roomie_opts* o, co
     fa.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u;
     fa.P_out = P_out; fa.evals_out = reinterpret_cast<unsigned long long*>(evals_out);
     // one CTA per pair: pairs differ in size by orders of magnitude, and the hardware hands the next pair
-    // to whichever SM frees a slot (a fixed stride per CTA was 30 % slower on the edge configuration)
-    uint32_t grid = ps.n_pairs;
+    // to whichever SM frees a slot (a fixed stride per CTA was 30 % slower on the edge configuration).  The
+    // grid lists every pair once per size class, largest class first; a CTA whose pair is of another class
+    // leaves at once, so the big tables start first and the small ones fill the tail.
+    uint64_t q1 = 0;
+    for (uint32_t p = 0; p < lib->num_profiles; ++p) {
+        const uint64_t q = lib->offsets_host[p + 1] - lib->offsets_host[p];
+        if (q > q1) q1 = q;
+    }
+    fa.max_cells = q1 * q1;
+    if ((uint64_t)ps.n_pairs * kFullClasses > 0x7fffffffull) return ROOMIE_ERR_CAPACITY;
+    uint32_t grid = ps.n_pairs * kFullClasses;
     profile_mark(st, true);
     lockstep_full_kernel<<<grid, kFullThreads, fa.n_inv * sizeof(float), st>>>(fa);
     profile_mark(st, false);

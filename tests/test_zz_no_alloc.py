@@ -45,6 +45,8 @@ def test_static_scratch_entry_point_matches_workspace_entry_point():
     # the runtime (module loading) or of torch's caching allocator
     rm.pair_interference_static(gl, 0, 1, detail_capacity=64, **calls[0][2])
     rm.pair_interference(gl, 0, 1, detail_capacity=64, **calls[0][2])
+    for _, _, kw in calls:                          # every kernel of every mode loaded once (the driver loads lazily)
+        rm.pair_interference_static(gl, 1, 0, **kw)
     torch.cuda.synchronize()
     # several calls in a row on the shared array, each compared with the workspace variant
     for a, b, kw in calls:
