@@ -408,17 +408,18 @@ def main():
         lane_peak = SM_COUNT * LANES_PER_SM * sm_hz                   # plain-ALU lane-instructions per second
         evals_rank = evals_per_step * ((pair_hi - pair_lo) / total_pairs)
         if args.setting == "lockstep_full":
-            # compute-bound kernel: table cells visited (q_a*q_b per pair and pass; the exact median takes 3
-            # passes, 4 when the number of kept alignments is even: 3 are counted) against the plain-ALU issue
-            # peak divided by the 53 lane-instructions one cell visit takes (ncu capture of configuration 2)
+            # compute-bound kernel: table cells visited (q_a*q_b per pair and pass; the exact median takes 2
+            # passes over the table when the values under its first digit fit the workspace's lists, as they
+            # do here) against the plain-ALU issue peak divided by the lane-instructions one cell visit takes
+            # (ncu capture of configuration 2)
             q = lib.q().astype(np.int64)
             ia, ib = np.triu_indices(P)
-            visits = 3.0 * float((q[ia] * q[ib]).sum())
-            peak_visits = lane_peak / 53.0 / 1e9
+            visits = 2.0 * float((q[ia] * q[ib]).sum())
+            peak_visits = lane_peak / 48.0 / 1e9
             ach = visits / kernel_s / 1e9 if walk_launches else None
             roofline = {"bound": "alu", "kernel": "lockstep_full_kernel", "achieved": ach, "peak": peak_visits,
                         "unit": "G cell visits/s", "frac": (ach / peak_visits) if ach else None,
-                        "peak_source": "derived: 148 SMs x 128 lanes x SM clock / 53 lane-instructions per visit",
+                        "peak_source": "derived: 148 SMs x 128 lanes x SM clock / 48 lane-instructions per visit",
                         "kernel_ms": per_launch_ms, "launches_per_step": launches_per_matrix, "traffic": None}
         elif args.setting == "lockstep":
             roofline = {"bound": "hbm", "kernel": "lockstep_tiles_kernel", "achieved": 32.0 * evals_rank / kernel_s / 1e9 / launches_per_matrix if walk_launches else None,

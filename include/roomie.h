@@ -189,7 +189,12 @@ typedef struct roomie_opts {
  * triangle: (0,0), (0,1), ..., (0,P-1), (1,1), ...; there are P(P+1)/2 of them. */
 
 /* Bytes of workspace that let roomie_pair_matrix process pairs [pair_begin, pair_end) in one
- * batch (a smaller workspace makes it split the range).  0 on invalid arguments. */
+ * batch (a smaller workspace makes it split the range).  0 on invalid arguments.
+ * For ROOMIE_WALK_LOCKSTEP with n_align = 0 the workspace is optional help, not a need: it holds
+ * the counter a persistent grid takes its pairs from and per-CTA lists of candidate values that
+ * save the exact median one of its three passes over a pair's table; the figure returned is what
+ * lets the library's largest tables use the lists (at most about 1.2 GB), any size >= 256 bytes
+ * is accepted and gives the same bits. */
 size_t roomie_pair_workspace_bytes(const roomie_library *lib /* host */, const roomie_opts *opts /* host */,
                                    uint64_t pair_begin, uint64_t pair_end);
 

@@ -6,39 +6,46 @@
 // at (s_i, s_j):  delta_i(s_i, s_j) = sum_t hit(s_i+t, s_j+t) * d_{s_i+t} * o_i/(o_i+o_j), so all
 // q_i*q_j alignments of a pair are the suffix sums along the q_i+q_j-1 diagonals of one q_i x q_j
 // table: q_i*q_j work instead of q_i*q_j*min(q).  The table is never stored: one thread walks four
-// neighbouring diagonals from their far ends and the values go
-// straight into the histogram of an exact radix select (3 digit passes of 11/11/10 bits over the
-// float bits, which order like the non-negative values - the first one also counts the kept
-// alignments).  For an even count the upper middle value comes out of the last digit pass as well: it is the same
-// value, the next occupied bin of the last histogram, or - when the lower middle is the largest value under its
-// 22-bit prefix - the smallest value above that prefix, which the pass tracks on the side.  Every pass recomputes the
-// suffix sums; a suffix sum is accumulated in double and ranked as float.
+// neighbouring diagonals from their far ends (a suffix sum is accumulated in double and ranked as float) and the
+// values go straight into an exact radix select over the float bits, which order like the non-negative values:
 //
-// One CTA per pair; both directions (delta_i, delta_j) are selected in the same passes.
+//   pass 1 over the table   histogram of the upper 13 bits; it also counts the kept alignments
+//   pass 2 over the table   the values that share the median's upper 13 bits (a few per cent of the table, their
+//                           number known from pass 1) are appended to a list in the CTA's part of the workspace
+//   two passes over the list  the next 10 and the last 9 bits
+//
+// When the list does not fit (no workspace, or a table dominated by one value) the last two digits are passes over
+// the table as well.  For an even count the upper middle value comes out of the last digit pass: it is the same
+// value, the next occupied bin of the last histogram, or the smallest value above the prefix, which the passes track
+// on the side.
+//
+// One CTA per pair, both directions (delta_i, delta_j) selected in the same passes.  With a workspace the grid is
+// persistent (two CTAs per SM) and takes the pairs from a counter, largest tables first.
 
 constexpr int kFullThreads = 512;
-constexpr int kFullBins = 2048;
+constexpr int kFullBits0 = 13, kFullBits1 = 10, kFullBits2 = 9;   // digits of the select, upper bits first
+constexpr int kFullBins = 1 << kFullBits0;                        // the widest histogram
+constexpr int kFullClasses = 4;                                   // size classes of the order of work, largest tables first
+constexpr uint32_t kFullMinList = 1024;                           // a list shorter than this per CTA and direction is not worth having
 
 struct FullArgs {
     LibView lib;
     PairSet ps;
     int start_filter;
-    const float* inv_table;       // 1/s, s <= 2W
-    uint32_t n_inv;
+    uint32_t n_inv;               // 2W + 1: the table of 1/s is built on chip
     float* P_out;
     unsigned long long* evals_out;
-    unsigned long long max_cells;  // upper bound of q_a * q_b over the pairs of the call (sets the size classes)
+    unsigned long long max_cells; // upper bound of q_a * q_b over the pairs of the call (sets the size classes)
+    uint32_t* work_counter;       // next item of work (zeroed by the host), or null: item = blockIdx.x
+    uint32_t* lists;              // [gridDim.x][2][list_cap] float bits, or null
+    uint32_t list_cap;
 };
-
-constexpr int kFullClasses = 4;   // size classes of the launch order, largest tables first
-
-enum FullPass : int { kPassDigit0 = 0, kPassDigit1 = 1, kPassDigit2 = 2 };
 
 struct FullSelect {               // state of the radix select of one direction
     uint32_t prefix;              // bits fixed so far
     uint32_t rank;                // rank still to find among the values that share the prefix
-    uint32_t value_bits;          // after digit 2: the element of rank k1 (the lower middle)
-    uint32_t upper_bits;          // after digit 2: the element of rank k1 + 1, if the count is even
+    uint32_t value_bits;          // after the last digit: the element of rank k1 (the lower middle)
+    uint32_t upper_bits;          // after the last digit: the element of rank k1 + 1, if the count is even
 };
 
 // walks every diagonal of the pair once; `visit(vi_bits, vj_bits, walk_len)` is called for every
@@ -52,20 +59,20 @@ constexpr int kDiags = 4;
 struct FullRec {                  // what a cell needs of one kernel
     uint32_t lo, hi;              // packed demand
     uint32_t w;                   // resident warps
-    float x;                      // duration in ticks * warps
+    double x;                     // duration in ticks * warps
 };
 
 __device__ __forceinline__ FullRec full_rec(const uint4& r) {
     FullRec f;
     f.lo = r.z; f.hi = r.w;
     f.w = r.z >> kWarpShift;
-    f.x = (float)(r.y - r.x) * small_int_to_float(f.w);
+    f.x = (double)((unsigned long long)(r.y - r.x) * f.w);
     return f;
 }
 
 template <class Visit>
 __device__ __forceinline__ void full_walk(const uint4* __restrict__ A, const uint4* __restrict__ B, uint32_t na,
-                                          uint32_t nb, PhiCap cap, const float* s_inv, int start_filter,
+                                          uint32_t nb, PhiCap cap, const double* s_inv, int start_filter,
                                           Visit visit) {
     const int32_t n_diag = (int32_t)(na + nb - 1);
     const int32_t n_groups = (n_diag + kDiags - 1) / kDiags;
@@ -93,9 +100,9 @@ __device__ __forceinline__ void full_walk(const uint4* __restrict__ A, const uin
                     ++len[m];
                     const bool hit = phi_exceeds(cap.lo - ra.lo, cap.hi - ra.hi, rb[m].lo, rb[m].hi);
                     if (hit) {
-                        const float inv = s_inv[ra.w + rb[m].w];
-                        si[m] += (double)(ra.x * inv);
-                        sj[m] += (double)(rb[m].x * inv);
+                        const double inv = s_inv[ra.w + rb[m].w];
+                        si[m] = fma(ra.x, inv, si[m]);
+                        sj[m] = fma(rb[m].x, inv, sj[m]);
                     }
                     if (!start_filter || hit) visit(__float_as_uint((float)si[m]), __float_as_uint((float)sj[m]), len[m]);
                 }
@@ -109,17 +116,19 @@ __device__ __forceinline__ void full_walk(const uint4* __restrict__ A, const uin
     }
 }
 
-// finds the bin that holds the element of rank `rank` in hist[0..kFullBins); every thread gets the
-// bin and the rank inside it.  s_scan: kFullThreads/32 + 2 words of shared scratch.
-// With `next_bin` the caller also learns whether the element of rank + 1 is in the same bin (next_bin = bin) or which
-// is the next occupied bin (kFullBins when there is none).
-__device__ __forceinline__ void full_locate(const uint32_t* hist, uint32_t rank, uint32_t* s_scan, uint32_t& bin,
-                                            uint32_t& rank_in_bin, uint32_t* next_bin = nullptr) {
-    constexpr int kPer = kFullBins / kFullThreads;                 // bins per thread
+// finds the bin that holds the element of rank `rank` in hist[0 .. 1 << bits); every thread gets the bin, the rank
+// inside it and the bin's count.  s_scan: kFullThreads/32 + 3 words of shared scratch.  With `next_bin` the caller
+// also learns whether the element of rank + 1 is in the same bin (next_bin = bin) or which is the next occupied
+// bin (1 << bits when there is none).
+__device__ __forceinline__ void full_locate(const uint32_t* hist, int bits, uint32_t rank, uint32_t* s_scan,
+                                            uint32_t& bin, uint32_t& rank_in_bin, uint32_t& count_in_bin,
+                                            uint32_t* next_bin = nullptr) {
+    const uint32_t nbins = 1u << bits;
+    const uint32_t per = (nbins + kFullThreads - 1) / kFullThreads;                // bins per thread
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    uint32_t h[kPer], mine = 0;
-#pragma unroll
-    for (int k = 0; k < kPer; ++k) { h[k] = hist[threadIdx.x * kPer + k]; mine += h[k]; }
+    const uint32_t first = threadIdx.x * per;
+    uint32_t mine = 0;
+    for (uint32_t k = 0; k < per; ++k) mine += first + k < nbins ? hist[first + k] : 0u;
     uint32_t incl = mine;
 #pragma unroll
     for (int s = 1; s < 32; s <<= 1) {
@@ -131,49 +140,190 @@ __device__ __forceinline__ void full_locate(const uint32_t* hist, uint32_t rank,
     uint32_t before = incl - mine;
     for (int w = 0; w < wid; ++w) before += s_scan[w];
     if (rank >= before && rank < before + mine) {                  // exactly one thread
-        uint32_t r = rank - before;
-        int k = 0;
-        while (r >= h[k]) { r -= h[k]; ++k; }
-        s_scan[kFullThreads / 32] = threadIdx.x * kPer + k;
+        uint32_t r = rank - before, k = first;
+        while (r >= hist[k]) { r -= hist[k]; ++k; }
+        s_scan[kFullThreads / 32] = k;
         s_scan[kFullThreads / 32 + 1] = r;
+        s_scan[kFullThreads / 32 + 2] = nbins;                      // next occupied bin, filled in below
     }
     __syncthreads();
     bin = s_scan[kFullThreads / 32];
     rank_in_bin = s_scan[kFullThreads / 32 + 1];
-    __syncthreads();
+    count_in_bin = hist[bin];
     if (next_bin) {
-        if (rank_in_bin + 1 < hist[bin]) *next_bin = bin;
+        if (rank_in_bin + 1 < count_in_bin) *next_bin = bin;
         else {
             // lowest occupied bin above `bin`: every thread proposes the first of its own bins, the minimum wins
-            if (threadIdx.x == 0) s_scan[kFullThreads / 32] = kFullBins;
-            __syncthreads();
-            uint32_t cand = kFullBins;
-#pragma unroll
-            for (int k = kPer - 1; k >= 0; --k) {
-                const uint32_t b = threadIdx.x * kPer + k;
-                if (b > bin && h[k]) cand = b;
+            uint32_t cand = nbins;
+            for (uint32_t k = per; k-- > 0;) {
+                const uint32_t b = first + k;
+                if (b < nbins && b > bin && hist[b]) cand = b;
             }
-            if (cand < (uint32_t)kFullBins) atomicMin(&s_scan[kFullThreads / 32], cand);
+            if (cand < nbins) atomicMin(&s_scan[kFullThreads / 32 + 2], cand);
             __syncthreads();
-            *next_bin = s_scan[kFullThreads / 32];
-            __syncthreads();
+            *next_bin = s_scan[kFullThreads / 32 + 2];
         }
     }
+    __syncthreads();
 }
 
-__global__ void __launch_bounds__(kFullThreads) lockstep_full_kernel(FullArgs g) {
-    __shared__ uint32_t s_hist[2][kFullBins];
-    __shared__ uint32_t s_scan[kFullThreads / 32 + 2];
-    __shared__ uint32_t s_gt[2];                     // per direction: smallest value above the 22-bit prefix
-    __shared__ unsigned long long s_ev;
-    __shared__ uint32_t s_n;
-    extern __shared__ float s_inv[];
+// appends v to the list; the lanes that come here together share one addition to the cursor
+__device__ __forceinline__ void full_append(uint32_t* list, uint32_t cap, uint32_t* cursor, uint32_t v) {
+    const uint32_t active = __activemask();
+    const int lane = threadIdx.x & 31, leader = __ffs(active) - 1;
+    uint32_t base = 0;
+    if (lane == leader) base = atomicAdd(cursor, (uint32_t)__popc(active));
+    base = __shfl_sync(active, base, leader);
+    const uint32_t at = base + __popc(active & ((1u << lane) - 1u));
+    if (at < cap) list[at] = v;
+}
 
-    // The grid is kFullClasses x n_pairs CTAs: CTA c * n_pairs + p takes pair p if the pair's table falls into size
-    // class c (class 0: at least a quarter of the largest possible table, then a factor of four per class) and
-    // leaves at once otherwise, so that the largest tables start first and the small ones fill the tail.
+struct FullShared {
+    uint32_t hist[2][kFullBins];
+    uint32_t scan[kFullThreads / 32 + 3];
+    uint32_t gt[2];               // per direction: smallest value above the prefix of the pass
+    uint32_t cursor[2];           // lengths of the two lists
+    uint32_t n;
+    uint32_t item;
+    unsigned long long ev;
+};
+
+__device__ __forceinline__ void full_clear(FullShared& sh, int bits) {
+    for (uint32_t i = threadIdx.x; i < (1u << bits); i += kFullThreads) { sh.hist[0][i] = 0; sh.hist[1][i] = 0; }
+    if (threadIdx.x == 0) { sh.gt[0] = sh.gt[1] = 0xffffffffu; sh.cursor[0] = sh.cursor[1] = 0; }
+}
+
+// the select of one pair; every thread of the CTA calls it
+__device__ __forceinline__ void full_pair(const FullArgs& g, FullShared& sh, const double* s_inv, uint32_t a,
+                                          uint32_t b, uint32_t offa, uint32_t offb, uint32_t na, uint32_t nb) {
+    const uint4* A = g.lib.records + offa;
+    const uint4* B = g.lib.records + offb;
+    FullSelect sel[2] = {};
+    // ---- pass 1 over the table: first digit, count, walk lengths
+    full_clear(sh, kFullBits0);
+    if (threadIdx.x == 0) { sh.ev = 0; sh.n = 0; }
+    __syncthreads();
     {
-        const uint32_t local = blockIdx.x % g.ps.n_pairs, cls = blockIdx.x / g.ps.n_pairs;
+        uint32_t cnt = 0;
+        unsigned long long ev = 0;
+        full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t len) {
+            ++cnt; ev += len;
+            atomicAdd(&sh.hist[0][vi >> (32 - kFullBits0)], 1u);
+            atomicAdd(&sh.hist[1][vj >> (32 - kFullBits0)], 1u);
+        });
+        atomicAdd(&sh.n, cnt);
+        atomicAdd(&sh.ev, ev);
+    }
+    __syncthreads();
+    const uint32_t n = sh.n;
+    if (threadIdx.x == 0 && g.evals_out && sh.ev) atomicAdd(g.evals_out, sh.ev);
+    if (n == 0) {                                                  // no alignment kept: both medians are zero
+        if (threadIdx.x == 0) store_pair_values(g.lib, g.ps, g.P_out, a, b, na, nb, 0.0f, 0.0f);
+        __syncthreads();
+        return;
+    }
+    uint32_t in_bin[2];
+    for (int dir = 0; dir < 2; ++dir) {
+        uint32_t bin, r;
+        full_locate(sh.hist[dir], kFullBits0, (n - 1) / 2, sh.scan, bin, r, in_bin[dir]);
+        sel[dir].prefix = bin; sel[dir].rank = r;
+    }
+    const bool listed = g.lists && in_bin[0] <= g.list_cap && in_bin[1] <= g.list_cap;
+    uint32_t* list_i = listed ? g.lists + (size_t)blockIdx.x * 2 * g.list_cap : nullptr;
+    uint32_t* list_j = listed ? list_i + g.list_cap : nullptr;
+    uint32_t above[2] = {0xffffffffu, 0xffffffffu};                // smallest table value above the first digit's bin
+    if (listed) {
+        // ---- pass 2 over the table: the values under the first digit's prefix go to the lists
+        full_clear(sh, 0);
+        __syncthreads();
+        const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
+        uint32_t gt_i = 0xffffffffu, gt_j = 0xffffffffu;
+        full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
+            const uint32_t ui = vi >> (32 - kFullBits0), uj = vj >> (32 - kFullBits0);
+            if (ui == pi) full_append(list_i, g.list_cap, &sh.cursor[0], vi); else if (ui > pi) gt_i = min(gt_i, vi);
+            if (uj == pj) full_append(list_j, g.list_cap, &sh.cursor[1], vj); else if (uj > pj) gt_j = min(gt_j, vj);
+        });
+        if (gt_i != 0xffffffffu) atomicMin(&sh.gt[0], gt_i);
+        if (gt_j != 0xffffffffu) atomicMin(&sh.gt[1], gt_j);
+        __syncthreads();
+        above[0] = sh.gt[0]; above[1] = sh.gt[1];
+        __syncthreads();
+    }
+    // ---- the two remaining digits: over the lists, or over the table again
+    for (int digit = 1; digit <= 2; ++digit) {
+        const int bits = digit == 1 ? kFullBits1 : kFullBits2;
+        const int low = digit == 1 ? kFullBits2 : 0;                // bits below this digit
+        const uint32_t mask = (1u << bits) - 1u;
+        full_clear(sh, bits);
+        __syncthreads();
+        const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
+        uint32_t gt_i = 0xffffffffu, gt_j = 0xffffffffu;
+        if (listed) {
+            for (uint32_t e = threadIdx.x; e < in_bin[0]; e += kFullThreads) {
+                const uint32_t v = list_i[e], u = v >> (low + bits);
+                if (u == pi) atomicAdd(&sh.hist[0][(v >> low) & mask], 1u); else if (u > pi) gt_i = min(gt_i, v);
+            }
+            for (uint32_t e = threadIdx.x; e < in_bin[1]; e += kFullThreads) {
+                const uint32_t v = list_j[e], u = v >> (low + bits);
+                if (u == pj) atomicAdd(&sh.hist[1][(v >> low) & mask], 1u); else if (u > pj) gt_j = min(gt_j, v);
+            }
+        } else {
+            full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
+                const uint32_t ui = vi >> (low + bits), uj = vj >> (low + bits);
+                if (ui == pi) atomicAdd(&sh.hist[0][(vi >> low) & mask], 1u); else if (ui > pi) gt_i = min(gt_i, vi);
+                if (uj == pj) atomicAdd(&sh.hist[1][(vj >> low) & mask], 1u); else if (uj > pj) gt_j = min(gt_j, vj);
+            });
+        }
+        if (gt_i != 0xffffffffu) atomicMin(&sh.gt[0], gt_i);
+        if (gt_j != 0xffffffffu) atomicMin(&sh.gt[1], gt_j);
+        __syncthreads();
+        for (int dir = 0; dir < 2; ++dir) {
+            uint32_t bin, r, cnt, next = 0;
+            full_locate(sh.hist[dir], bits, sel[dir].rank, sh.scan, bin, r, cnt, digit == 2 ? &next : nullptr);
+            const uint32_t group = sel[dir].prefix;                  // the bits fixed before this pass
+            sel[dir].prefix = (group << bits) | bin;
+            sel[dir].rank = r;
+            if (digit == 2) {
+                // the element of rank + 1: same value, next occupied bin, smallest value above the prefix of this
+                // pass (over the list that is only the part under the first digit: the table's comes after it)
+                sel[dir].value_bits = sel[dir].prefix;
+                const uint32_t gt = sh.gt[dir] != 0xffffffffu ? sh.gt[dir] : above[dir];
+                sel[dir].upper_bits = next <= mask ? ((group << bits) | next) : gt;
+            }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        float med[2];
+        for (int dir = 0; dir < 2; ++dir) {
+            const float lo = __uint_as_float(sel[dir].value_bits);
+            const float hi = (n & 1u) ? lo : __uint_as_float(sel[dir].upper_bits);   // odd count: one middle
+            med[dir] = 0.5f * (lo + hi);
+        }
+        store_pair_values(g.lib, g.ps, g.P_out, a, b, na, nb, med[0], med[1]);
+    }
+    __syncthreads();
+}
+
+// Items of work: item c * n_pairs + p is pair p if the pair's table falls into size class c (class 0: at least a
+// quarter of the largest possible table, then a factor of four per class) and nothing otherwise, so that the largest
+// tables start first and the small ones fill the tail.
+__global__ void __launch_bounds__(kFullThreads, 2) lockstep_full_kernel(FullArgs g) {
+    extern __shared__ __align__(16) unsigned char full_smem[];
+    FullShared& sh = *reinterpret_cast<FullShared*>(full_smem);
+    double* s_inv = reinterpret_cast<double*>(full_smem + sizeof(FullShared));   // 1/s, s = 1 .. 2W (0 never interferes)
+    for (uint32_t i = threadIdx.x; i < g.n_inv; i += kFullThreads) s_inv[i] = i ? 1.0 / (double)i : 0.0;
+    __syncthreads();
+    const unsigned long long n_items = (unsigned long long)kFullClasses * g.ps.n_pairs;
+    for (unsigned long long item = blockIdx.x;; item += gridDim.x) {
+        if (g.work_counter) {
+            if (threadIdx.x == 0) sh.item = atomicAdd(g.work_counter, 1u);
+            __syncthreads();
+            item = sh.item;
+            __syncthreads();
+        }
+        if (item >= n_items) break;
+        const uint32_t local = (uint32_t)(item % g.ps.n_pairs), cls = (uint32_t)(item / g.ps.n_pairs);
         uint32_t a, b;
         pair_of(g.ps, g.lib.P, local, a, b);
         const uint32_t offa = g.lib.offsets[a], offb = g.lib.offsets[b];
@@ -183,77 +333,6 @@ __global__ void __launch_bounds__(kFullThreads) lockstep_full_kernel(FullArgs g)
 #pragma unroll
         for (int c = kFullClasses - 2; c >= 0; --c)
             if (cells >= (g.max_cells >> (2 * c + 2))) mine = c;
-        if (mine != cls) return;
-        for (uint32_t i = threadIdx.x; i < g.n_inv; i += kFullThreads) s_inv[i] = __ldg(&g.inv_table[i]);
-        const uint4* A = g.lib.records + offa;
-        const uint4* B = g.lib.records + offb;
-        FullSelect sel[2] = {};
-        uint32_t n = 0;
-        for (int pass = kPassDigit0; pass <= kPassDigit2; ++pass) {
-            for (uint32_t i = threadIdx.x; i < 2 * kFullBins; i += kFullThreads) (&s_hist[0][0])[i] = 0;
-            if (threadIdx.x == 0) { s_ev = 0; s_n = 0; s_gt[0] = s_gt[1] = 0xffffffffu; }
-            __syncthreads();
-            if (pass == kPassDigit0) {                                   // first digit, count and walk lengths
-                uint32_t cnt = 0;
-                unsigned long long ev = 0;
-                full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t len) {
-                    ++cnt; ev += len;
-                    atomicAdd(&s_hist[0][vi >> 21], 1u);
-                    atomicAdd(&s_hist[1][vj >> 21], 1u);
-                });
-                atomicAdd(&s_n, cnt);
-                atomicAdd(&s_ev, ev);
-            } else if (pass == kPassDigit1) {
-                const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
-                full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
-                    if ((vi >> 21) == pi) atomicAdd(&s_hist[0][(vi >> 10) & 2047u], 1u);
-                    if ((vj >> 21) == pj) atomicAdd(&s_hist[1][(vj >> 10) & 2047u], 1u);
-                });
-            } else {
-                // last digit; on the side, the smallest value whose upper 22 bits lie above the prefix (the upper
-                // middle of an even count when the lower middle is the largest value under the prefix)
-                const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
-                uint32_t gt_i = 0xffffffffu, gt_j = 0xffffffffu;
-                full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
-                    const uint32_t ui = vi >> 10, uj = vj >> 10;
-                    if (ui == pi) atomicAdd(&s_hist[0][vi & 1023u], 1u); else if (ui > pi) gt_i = min(gt_i, vi);
-                    if (uj == pj) atomicAdd(&s_hist[1][vj & 1023u], 1u); else if (uj > pj) gt_j = min(gt_j, vj);
-                });
-                if (gt_i != 0xffffffffu) atomicMin(&s_gt[0], gt_i);
-                if (gt_j != 0xffffffffu) atomicMin(&s_gt[1], gt_j);
-            }
-            __syncthreads();
-            if (pass == kPassDigit0) {
-                n = s_n;
-                if (threadIdx.x == 0 && g.evals_out && s_ev) atomicAdd(g.evals_out, s_ev);
-                if (n == 0) break;
-                sel[0].rank = sel[1].rank = (n - 1) / 2;
-            }
-            const int bits = pass == kPassDigit2 ? 10 : 11;
-            for (int dir = 0; dir < 2; ++dir) {
-                uint32_t bin, r, next = 0;
-                full_locate(s_hist[dir], sel[dir].rank, s_scan, bin, r, pass == kPassDigit2 ? &next : nullptr);
-                const uint32_t group = sel[dir].prefix;                  // the bits fixed before this pass
-                sel[dir].prefix = (group << bits) | bin;
-                sel[dir].rank = r;
-                if (pass == kPassDigit2) {
-                    sel[dir].value_bits = sel[dir].prefix;
-                    sel[dir].upper_bits = next < (uint32_t)kFullBins ? ((group << 10) | next) : s_gt[dir];
-                }
-            }
-            __syncthreads();
-        }
-        if (threadIdx.x == 0) {
-            float med[2] = {0.0f, 0.0f};
-            if (n > 0) {
-                for (int dir = 0; dir < 2; ++dir) {
-                    const float lo = __uint_as_float(sel[dir].value_bits);
-                    const float hi = (n & 1u) ? lo : __uint_as_float(sel[dir].upper_bits);   // odd count: one middle
-                    med[dir] = 0.5f * (lo + hi);
-                }
-            }
-            store_pair_values(g.lib, g.ps, g.P_out, a, b, na, nb, med[0], med[1]);
-        }
-        __syncthreads();
+        if (mine == cls) full_pair(g, sh, s_inv, a, b, offa, offb, na, nb);
     }
 }

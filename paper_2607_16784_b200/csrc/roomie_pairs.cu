@@ -691,9 +691,31 @@ static int slots_for(const roomie_library* lib, const roomie_opts* o, bool expli
     return ROOMIE_OK;
 }
 
-// Algorithm 1 as printed with the full Cartesian alignment set: no scratch, one CTA per pair
+// Algorithm 1 as printed with the full Cartesian alignment set, one CTA per pair.  With a workspace the grid is
+// persistent: the workspace holds the counter the CTAs take their pairs from and, per CTA and direction, a list for
+// the values under the median's first digit.  Without one (or with one too small for useful lists) every pass goes
+// over the table and the grid has one CTA per item of work.
+static uint32_t full_ctas() { return 2u * (uint32_t)sm_count(); }
+static size_t full_smem_bytes(const roomie_library* lib) {
+    return sizeof(FullShared) + (2u * (lib->spec.threads_per_sm / 32u) + 1u) * sizeof(double);
+}
+static uint64_t largest_table(const roomie_library* lib) {
+    uint64_t q1 = 0;
+    for (uint32_t p = 0; p < lib->num_profiles; ++p) {
+        const uint64_t q = lib->offsets_host[p + 1] - lib->offsets_host[p];
+        if (q > q1) q1 = q;
+    }
+    return q1 * q1;
+}
+// what lets every pair of the library use the lists, within a fixed bound
+static size_t full_workspace_bytes(const roomie_library* lib) {
+    uint64_t cap = largest_table(lib) / 8 + kFullMinList;           // the first digit's bin holds a few per cent
+    if (cap > (1u << 19)) cap = 1u << 19;
+    return 256 + (size_t)full_ctas() * 2 * cap * sizeof(uint32_t);
+}
+
 static int run_lockstep_full(const roomie_library* lib, const roomie_opts* o, const PairSet& ps, float* P_out,
-                             uint64_t* evals_out, cudaStream_t st) {
+                             uint64_t* evals_out, void* workspace, size_t workspace_bytes, cudaStream_t st) {
     FullArgs fa;
     fa.lib.records = static_cast<const uint4*>(lib->records);
     fa.lib.offsets = lib->offsets;
@@ -701,23 +723,35 @@ static int run_lockstep_full(const roomie_library* lib, const roomie_opts* o, co
     fa.lib.P = lib->num_profiles;
     fa.lib.cap = make_cap(lib->spec);
     fa.ps = ps; fa.start_filter = o->start_filter;
-    fa.inv_table = lib->share_table;
     fa.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u;
     fa.P_out = P_out; fa.evals_out = reinterpret_cast<unsigned long long*>(evals_out);
-    // one CTA per pair: pairs differ in size by orders of magnitude, and the hardware hands the next pair
-    // to whichever SM frees a slot (a fixed stride per CTA was 30 % slower on the edge configuration).  The
-    // grid lists every pair once per size class, largest class first; a CTA whose pair is of another class
-    // leaves at once, so the big tables start first and the small ones fill the tail.
-    uint64_t q1 = 0;
-    for (uint32_t p = 0; p < lib->num_profiles; ++p) {
-        const uint64_t q = lib->offsets_host[p + 1] - lib->offsets_host[p];
-        if (q > q1) q1 = q;
+    fa.max_cells = largest_table(lib);
+    const uint64_t items = (uint64_t)ps.n_pairs * kFullClasses;
+    if (items > 0x7fffffffull) return ROOMIE_ERR_CAPACITY;
+    uint32_t grid = (uint32_t)items;
+    fa.work_counter = nullptr; fa.lists = nullptr; fa.list_cap = 0;
+    const uint32_t ctas = full_ctas() < grid ? full_ctas() : grid;
+    if (workspace && workspace_bytes >= 256 + (size_t)ctas * 2 * kFullMinList * sizeof(uint32_t)) {
+        uint64_t cap = (workspace_bytes - 256) / ((size_t)ctas * 2 * sizeof(uint32_t));
+        if (cap > 0x7fffffffull) cap = 0x7fffffffull;
+        fa.work_counter = static_cast<uint32_t*>(workspace);
+        fa.lists = reinterpret_cast<uint32_t*>(static_cast<unsigned char*>(workspace) + 256);
+        fa.list_cap = (uint32_t)cap;
+        grid = ctas;
+        ROOMIE_CUDA_OK(cudaMemsetAsync(fa.work_counter, 0, sizeof(uint32_t), st));
     }
-    fa.max_cells = q1 * q1;
-    if ((uint64_t)ps.n_pairs * kFullClasses > 0x7fffffffull) return ROOMIE_ERR_CAPACITY;
-    uint32_t grid = ps.n_pairs * kFullClasses;
+    const size_t smem = full_smem_bytes(lib);
+    static thread_local int smem_set_for = -1;
+    int dev = 0;
+    ROOMIE_CUDA_OK(cudaGetDevice(&dev));
+    if (smem_set_for != dev) {
+        ROOMIE_CUDA_OK(cudaFuncSetAttribute(lockstep_full_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)(sizeof(FullShared) + 4096)));
+        smem_set_for = dev;
+    }
+    if (smem > sizeof(FullShared) + 4096) return ROOMIE_ERR_CAPACITY;
     profile_mark(st, true);
-    lockstep_full_kernel<<<grid, kFullThreads, fa.n_inv * sizeof(float), st>>>(fa);
+    lockstep_full_kernel<<<grid, kFullThreads, smem, st>>>(fa);
     profile_mark(st, false);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
@@ -916,7 +950,7 @@ extern "C" size_t roomie_pair_workspace_bytes(const roomie_library* lib, const r
     const uint64_t total = (uint64_t)lib->num_profiles * (lib->num_profiles + 1) / 2;
     if (pair_end > total) pair_end = total;
     if (pair_begin >= pair_end) return 0;
-    if (wants_lockstep_full(opts)) return 256;                       // that path keeps everything on chip
+    if (wants_lockstep_full(opts)) return full_workspace_bytes(lib);
     uint32_t slots;
     if (slots_for(lib, opts, false, 0, 0, slots) != ROOMIE_OK) return 0;
     Need need;
@@ -950,7 +984,7 @@ extern "C" int roomie_pair_matrix(const roomie_library* lib, const roomie_opts* 
         if (pair_end - pair_begin >= (1ull << 31)) return ROOMIE_ERR_CAPACITY;
         PairSet ps;
         ps.pair_begin = pair_begin; ps.n_pairs = (uint32_t)(pair_end - pair_begin); ps.explicit_pair = 0; ps.a = ps.b = 0;
-        return run_lockstep_full(lib, opts, ps, P_out, evals_out, st);
+        return run_lockstep_full(lib, opts, ps, P_out, evals_out, workspace, workspace_bytes, st);
     }
     uint32_t slots;
     rc = slots_for(lib, opts, false, 0, 0, slots);
@@ -989,7 +1023,7 @@ extern "C" int roomie_pair_interference(const roomie_library* lib, uint32_t a, u
     if (wants_lockstep_full(opts) && !detail) {
         PairSet fps;
         fps.pair_begin = 0; fps.n_pairs = 1; fps.explicit_pair = 1; fps.a = a; fps.b = b;
-        return run_lockstep_full(lib, opts, fps, out2, evals_out, st);
+        return run_lockstep_full(lib, opts, fps, out2, evals_out, workspace, workspace_bytes, st);
     }
     uint32_t slots;
     rc = slots_for(lib, opts, true, a, b, slots);
@@ -1013,7 +1047,7 @@ extern "C" int roomie_pair_interference_static(const roomie_library* lib, uint32
         if (evals_out) ROOMIE_CUDA_OK(cudaMemsetAsync(evals_out, 0, sizeof(uint64_t), fst));
         PairSet fps;
         fps.pair_begin = 0; fps.n_pairs = 1; fps.explicit_pair = 1; fps.a = a; fps.b = b;
-        return run_lockstep_full(lib, opts, fps, out2, evals_out, fst);
+        return run_lockstep_full(lib, opts, fps, out2, evals_out, nullptr, 0, fst);
     }
     uint32_t slots;
     rc = slots_for(lib, opts, true, a, b, slots);

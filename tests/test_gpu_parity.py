@@ -568,6 +568,30 @@ def test_lockstep_full_cartesian_long_profiles_and_special_cases(rm, oracle):
         assert r["P2"].cpu().tolist() == [0.0, 0.0] and int(r["evals"].item()) == (0 if sf else sum(min(30 - i, 20 - j) for i in range(30) for j in range(20)))
 
 
+def test_lockstep_full_cartesian_lists_and_table_passes_agree(rm):
+    """The exact median of the full alignment set comes out the same whatever the workspace allows: with lists of
+    the values under the median's first digit (large workspace), with passes over the table only (lists too short
+    for those values, or no lists at all), on a persistent grid or with one CTA per item of work.  (Parity with the
+    oracle in this mode: the tests above, which run with the default workspace and so with lists.)"""
+    import torch
+    lib = rs.make_library(2)
+    gl = rm.library_build(lib.grid_blocks, lib.block_threads, lib.regs_per_thread, lib.smem_per_block,
+                          lib.dur_us, lib.gap_us, lib.offsets, lib.spec)
+    big = torch.zeros(512 << 20, dtype=torch.uint8, device="cuda")
+    # 2 CTAs per SM x 2 directions x 1100 values: lists exist, but most pairs' first-digit bins do not fit them
+    small = torch.zeros(256 + 2 * 148 * 2 * 1100 * 4, dtype=torch.uint8, device="cuda")
+    tiny = torch.zeros(256, dtype=torch.uint8, device="cuda")           # no lists, no counter
+    for sf in (0, 1):
+        kw = dict(mode=1, n_align=0, start_filter=sf, pair_end=40)
+        got_big, ev_big = rm.pair_matrix(gl, workspace=big, **kw)
+        got_small, ev_small = rm.pair_matrix(gl, workspace=small, **kw)
+        got_tiny, ev_tiny = rm.pair_matrix(gl, workspace=tiny, **kw)
+        assert int(ev_big.item()) == int(ev_small.item()) == int(ev_tiny.item()) > 0
+        assert torch.equal(got_big, got_small) and torch.equal(got_big, got_tiny)
+        assert int((got_big > 0).sum().item()) >= 40
+    assert gl.status_flags() == 0
+
+
 # ----------------------------------------------------------------------------- optimal deployment search
 def test_optimal_assignment_bit_exact(rm, oracle):
     rng = np.random.default_rng(3)
