@@ -231,22 +231,15 @@ __device__ __forceinline__ void full_pair(const FullArgs& g, FullShared& sh, con
     const bool listed = g.lists && in_bin[0] <= g.list_cap && in_bin[1] <= g.list_cap;
     uint32_t* list_i = listed ? g.lists + (size_t)blockIdx.x * 2 * g.list_cap : nullptr;
     uint32_t* list_j = listed ? list_i + g.list_cap : nullptr;
-    uint32_t above[2] = {0xffffffffu, 0xffffffffu};                // smallest table value above the first digit's bin
     if (listed) {
         // ---- pass 2 over the table: the values under the first digit's prefix go to the lists
         full_clear(sh, 0);
         __syncthreads();
         const uint32_t pi = sel[0].prefix, pj = sel[1].prefix;
-        uint32_t gt_i = 0xffffffffu, gt_j = 0xffffffffu;
         full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
-            const uint32_t ui = vi >> (32 - kFullBits0), uj = vj >> (32 - kFullBits0);
-            if (ui == pi) full_append(list_i, g.list_cap, &sh.cursor[0], vi); else if (ui > pi) gt_i = min(gt_i, vi);
-            if (uj == pj) full_append(list_j, g.list_cap, &sh.cursor[1], vj); else if (uj > pj) gt_j = min(gt_j, vj);
+            if ((vi >> (32 - kFullBits0)) == pi) full_append(list_i, g.list_cap, &sh.cursor[0], vi);
+            if ((vj >> (32 - kFullBits0)) == pj) full_append(list_j, g.list_cap, &sh.cursor[1], vj);
         });
-        if (gt_i != 0xffffffffu) atomicMin(&sh.gt[0], gt_i);
-        if (gt_j != 0xffffffffu) atomicMin(&sh.gt[1], gt_j);
-        __syncthreads();
-        above[0] = sh.gt[0]; above[1] = sh.gt[1];
         __syncthreads();
     }
     // ---- the two remaining digits: over the lists, or over the table again
@@ -285,12 +278,30 @@ __device__ __forceinline__ void full_pair(const FullArgs& g, FullShared& sh, con
             sel[dir].rank = r;
             if (digit == 2) {
                 // the element of rank + 1: same value, next occupied bin, smallest value above the prefix of this
-                // pass (over the list that is only the part under the first digit: the table's comes after it)
+                // pass (none: all ones; over the list that is only the part under the first digit, see below)
                 sel[dir].value_bits = sel[dir].prefix;
-                const uint32_t gt = sh.gt[dir] != 0xffffffffu ? sh.gt[dir] : above[dir];
-                sel[dir].upper_bits = next <= mask ? ((group << bits) | next) : gt;
+                sel[dir].upper_bits = next <= mask ? ((group << bits) | next) : sh.gt[dir];
             }
         }
+        __syncthreads();
+    }
+    if (listed && !(n & 1u) && (sel[0].upper_bits == 0xffffffffu || sel[1].upper_bits == 0xffffffffu)) {
+        // the lower middle is the largest value under its first digit, so the upper middle is not in the list: it is
+        // the smallest value of the table above that digit's bin (one more pass; with thousands of values per bin
+        // this hardly ever happens)
+        full_clear(sh, 0);
+        __syncthreads();
+        const uint32_t pi = sel[0].value_bits >> (32 - kFullBits0), pj = sel[1].value_bits >> (32 - kFullBits0);
+        uint32_t gt_i = 0xffffffffu, gt_j = 0xffffffffu;
+        full_walk(A, B, na, nb, g.lib.cap, s_inv, g.start_filter, [&](uint32_t vi, uint32_t vj, uint32_t) {
+            if ((vi >> (32 - kFullBits0)) > pi) gt_i = min(gt_i, vi);
+            if ((vj >> (32 - kFullBits0)) > pj) gt_j = min(gt_j, vj);
+        });
+        if (gt_i != 0xffffffffu) atomicMin(&sh.gt[0], gt_i);
+        if (gt_j != 0xffffffffu) atomicMin(&sh.gt[1], gt_j);
+        __syncthreads();
+        for (int dir = 0; dir < 2; ++dir)
+            if (sel[dir].upper_bits == 0xffffffffu) sel[dir].upper_bits = sh.gt[dir];
         __syncthreads();
     }
     if (threadIdx.x == 0) {

@@ -558,6 +558,19 @@ def test_lockstep_full_cartesian_long_profiles_and_special_cases(rm, oracle):
         assert got[0] == pytest.approx(max(qa / qb, 1.0) * med / (qa * 50000.0), rel=1e-6)
         want = oracle.pair(ol2, 0, 1, mode=1, n_align=0, cap_align=1)
         assert_close(got, [want.P_ab, want.P_ba])
+    # an even count whose two middle values differ by more than the select's first digit resolves: the upper one is
+    # then not among the listed candidates and is fetched by the extra pass over the table
+    for durs in ((10000, 30000), (10000, 10500, 40000, 90000)):
+        lib4 = make_lib([[(256, 64, 0, d, 0.05, 0.0) for d in durs], [k]])
+        ol4 = oracle.library_build(lib4)
+        gl4 = rm.library_build(lib4.grid_blocks, lib4.block_threads, lib4.regs_per_thread, lib4.smem_per_block,
+                               lib4.dur_us, lib4.gap_us, lib4.offsets, lib4.spec)
+        for x, y in ((0, 1), (1, 0)):
+            want = oracle.pair(ol4, x, y, mode=1, n_align=0, cap_align=1)
+            got = rm.pair_interference(gl4, x, y, mode=1, n_align=0)
+            assert_close(got["P2"].cpu().numpy(), [want.P_ab, want.P_ba])
+            st = rm.pair_interference_static(gl4, x, y, mode=1, n_align=0)
+            assert np.array_equal(st["P2"].cpu().numpy(), got["P2"].cpu().numpy())
     # nothing interferes: kept set empty under the filter, all delays zero without it
     small = (64, 16, 0, 100, 0.01, 0.001)
     lib3 = make_lib([[small] * 30, [small] * 20])
