@@ -71,7 +71,48 @@ struct PlaceArgs {
     int admit_rule;         // 0: mean drop < lambda, 1: largest member drop < lambda
     int objective;          // 0: lowest mean drop, 1: lowest largest drop, 2: lowest drop of the arrival
     uint32_t chunk;         // fast kernel: arrivals staged in shared memory at a time (<= kArrChunk)
+    // A long single stream is served by whichever of two kernels suits its admission rate (see place_impl): the
+    // kernels are launched in turn, and the one that is running hands the rest of the stream to the next launch
+    // when the other kind has become the faster one.
+    int32_t* mailbox;        // where a kernel leaves the hand-over for the next launch (the stream's last gpu_out
+                             // element, which holds a decision once the stream is done), or null
+    int32_t my_kind;         // 0: one lane per modelled GPU, 1: one lane per resident slot
+    int32_t first;           // 1: the first launch (starts at arrival 0 without looking at the mailbox)
+    int32_t may_hand_over;   // 0: the last launch (finishes the stream whatever the admission rate)
 };
+
+constexpr uint32_t kPlaceAdaptiveFrom = 4096;      // arrivals from which a single stream may change kernels
+constexpr uint32_t kPlaceWindow = 1024;            // arrivals between two looks at the admission rate
+constexpr int kPlaceLaunches = 5;                  // launches of such a stream: kinds 1, 0, 1, 0, 1
+// hand-over word: -100 - 2 * (arrivals done / kPlaceWindow) - kind of the kernel that continues (decisions are >= -3)
+__device__ __forceinline__ int32_t hand_over_word(uint32_t done, int32_t kind) {
+    return -100 - 2 * (int32_t)(done / kPlaceWindow) - kind;
+}
+// where this launch starts: false = nothing to do (the stream is done, or the hand-over names the other kind)
+__device__ __forceinline__ bool place_start(const PlaceArgs& g, uint32_t& k_begin) {
+    k_begin = 0;
+    if (!g.mailbox || g.first) return true;
+    const int32_t m = g.mailbox[0];
+    if (m > -100 || ((-100 - m) & 1) != g.my_kind) return false;
+    k_begin = (uint32_t)((-100 - m) >> 1) * kPlaceWindow;
+    return true;
+}
+// which kind suits the admissions of the last window: one lane per GPU is the faster one while fewer than about
+// half of the arrivals are admitted (its cost grows with the admissions), one lane per slot beyond that
+__device__ __forceinline__ int32_t kind_for(uint32_t placed, uint32_t n, int32_t mine) {
+    if (placed * 100ull < 45ull * n) return 0;
+    if (placed * 100ull > 55ull * n) return 1;
+    return mine;
+}
+// sum of `mine` over the CTA, for thread 0 (s_word: a shared word nobody else uses)
+__device__ __forceinline__ uint32_t block_count(uint32_t mine, uint32_t* s_word) {
+    if (threadIdx.x == 0) *s_word = 0;
+    __syncthreads();
+    mine = __reduce_add_sync(0xffffffffu, mine);
+    if ((threadIdx.x & 31) == 0 && mine) atomicAdd(s_word, mine);
+    __syncthreads();
+    return *s_word;
+}
 
 constexpr unsigned long long kNoGpu = ~0ull;
 
@@ -377,6 +418,11 @@ __device__ __forceinline__ void cp_async_4_s(uint32_t smem_addr, const void* gme
 template <bool kPlain>
 __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
     select_stream(g);
+    uint32_t k_begin;
+    if (!place_start(g, k_begin)) return;                                   // not this launch's turn
+    __shared__ uint32_t s_placed;
+    uint32_t n_placed = 0;                                                  // admissions since the last look
+    uint32_t k_end = g.n;                                                   // where this launch stops
     // one float/int array; every region is addressed by a 32-bit word index
     extern __shared__ __align__(16) float sm[];
     int32_t* smi = reinterpret_cast<int32_t*>(sm);
@@ -445,7 +491,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
         }
         pub[gpu] = (unsigned long long)ord | ((unsigned long long)c << 32);
     }
-    const uint32_t tick0 = *g.tick;
+    const uint32_t tick0 = *g.tick - k_begin;                               // tick of the stream's first arrival
 
     // fetch warps: what arrival a (staged index a_local, global index a_global) will need
     auto issue = [&](uint32_t a_local, uint32_t a_global) {
@@ -474,22 +520,25 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
         }
     };
 
-    for (uint32_t k0 = 0; k0 < g.n; k0 += chunk) {
+    for (uint32_t k0 = k_begin; k0 < g.n; k0 += chunk) {
         const uint32_t kn = min(chunk, g.n - k0);
         // stage arrival ids [k0 - kLead, k0 + kn + kLead) and lifetimes [k0, k0 + kn)
         __syncthreads();
+        bool saw_bad = false;
         for (uint32_t i = tid; i < kn + 2 * kLead; i += blockDim.x) {
             const long long gi = (long long)k0 + i - kLead;
             int32_t id = 0;
-            if (gi >= 0 && gi < (long long)g.n) { id = g.arr_id[gi]; if ((uint32_t)id >= P) id = -1; }
+            if (gi >= 0 && gi < (long long)g.n) { id = g.arr_id[gi]; if ((uint32_t)id >= P) { id = -1; saw_bad = true; } }
             smi[oARR + i] = id;
         }
         for (uint32_t i = tid; i < kn; i += blockDim.x) smi[oLIFE + i] = (int32_t)g.arr_life[k0 + i];
-        __syncthreads();
-        if (k0 == 0) {                                                      // prime: arrivals 0 .. kAhead-1
+        // whether the chunk holds an id outside the matrix at all: the per-arrival look at the staged id would
+        // otherwise sit on every arrival's chain
+        const bool chunk_bad = __syncthreads_or(saw_bad);
+        if (k0 == k_begin) {                                                // prime: the first kAhead arrivals of this launch
             if (fetcher) {
                 for (uint32_t a = 0; a < (uint32_t)kAhead; ++a) {
-                    if (a < g.n) issue(a + kLead, a);
+                    if (k_begin + a < g.n) issue(a + kLead, k_begin + a);
                     cp_async_commit();
                 }
                 cp_async_wait<kAhead - 1>();
@@ -529,8 +578,7 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             const uint32_t young_k = oYOUNG + (kg & (kYoungRing - 1)) * kYoungD * 2;
             uint32_t key_hi = 0xffffffffu;
             float mean = 0.0f, mu_inc = 0.0f;
-            const bool bad_arrival = smi[oARR + kl] < 0;
-            if (owner && c < R && !bad_arrival) {                            // what-if: residents + the arrival
+            if (owner && c < R) {                                            // what-if: residents + the arrival
                 float tot = 0.0f, worst = 0.0f;
                 // two-stage pipeline over the residents: while resident t is summed, the terms of t + 1 are on
                 // their way and the birth index and cached partial sum of t + 2 are being read (past the end
@@ -571,6 +619,13 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
                 mean = div_small(tot, c + 1);                                // c + 1 <= 9 in this kernel
                 key_hi = kPlain ? (mean < g.lambda ? __float_as_uint(mean) : 0xffffffffu)
                                 : decision_key(g, mean, fmaxf(worst, mu_inc), mu_inc);
+            }
+            // an arrival whose id is outside the matrix (staged as -1, its terms fetched for profile 0) goes nowhere;
+            // the look at the staged id is skipped for a chunk without such ids, which keeps it off the chain
+            bool bad_arrival = false;
+            if (chunk_bad) {
+                bad_arrival = smi[oARR + kl] < 0;
+                if (bad_arrival) key_hi = 0xffffffffu;
             }
             // warp argmin: lowest key, then the lowest lane (= lowest GPU index of this warp) that holds it
             const uint32_t best_hi = __reduce_min_sync(0xffffffffu, key_hi);
@@ -617,8 +672,16 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
         __syncthreads();
         for (uint32_t i = tid; i < kn; i += blockDim.x) {
             g.gpu_out[k0 + i] = smi[oOUT + i];
+            n_placed += smi[oOUT + i] >= 0 ? 1u : 0u;
             if (g.mean_out) g.mean_out[k0 + i] = sm[oOUT + chunk + i];
             if (g.mu_arr_out) g.mu_arr_out[k0 + i] = sm[oOUT + 2 * chunk + i];
+        }
+        // a look at the admission rate: should the other kind of kernel take the rest of the stream?
+        const uint32_t done = k0 + kn;
+        if (g.mailbox && g.may_hand_over && done < g.n && done % kPlaceWindow == 0) {
+            const uint32_t placed = block_count(n_placed, &s_placed);
+            n_placed = 0;
+            if (kind_for(placed, kn, g.my_kind) != g.my_kind) { k_end = done; break; }
         }
     }
     cp_async_wait<0>();
@@ -630,7 +693,10 @@ __global__ void __launch_bounds__(1024) place_fast_kernel(PlaceArgs g) {
             g.expiry[gpu * R + t] = t < c ? smu[oEX + p * G] : 0u;
         }
     }
-    if (tid == 0) *g.tick = tick0 + g.n;
+    if (tid == 0) {
+        *g.tick = tick0 + k_end;
+        if (k_end < g.n) g.mailbox[0] = hand_over_word(k_end, 1 - g.my_kind);
+    }
 }
 
 #include "roomie_place_slots.cuh"
@@ -672,18 +738,45 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
     a.arr_id = arr_id; a.arr_life = arr_life; a.n = n; a.lambda = opts->lambda;
     a.gpu_out = gpu_out; a.mean_out = mean_out; a.mu_arr_out = mu_arr_out;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    a.mailbox = nullptr; a.my_kind = 0; a.first = 1; a.may_hand_over = 0;
+    const bool plain = a.admit_rule == 0 && a.objective == 0;
     if (num_streams == 1 && a.R <= (uint32_t)kSlotLanes && a.G <= (1024u - 32u) / kSlotLanes) {
-        // one stream, up to 8 slots per GPU: one lane per resident slot (the shortest dependent chain; a batch of
-        // independent streams is a throughput problem and takes the one-lane-per-GPU kernel below instead)
-        a.matrix_mode = 1; a.pair_cache = 1; a.gpus_per_warp = 32 / kSlotLanes; a.chunk = kSlotChunk;
-        const uint32_t threads = ((a.G * kSlotLanes + 31) / 32) * 32 + 32;   // one more warp that owns no GPU
-        const size_t bytes = (size_t)slot_layout(threads, a.G).total * sizeof(float);
-        auto kern = (a.admit_rule == 0 && a.objective == 0) ? place_slots_kernel<true> : place_slots_kernel<false>;
-        if (bytes > 48 * 1024)
-            ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-        kern<<<1, threads, bytes, st>>>(a);
-        note_launch();
-        ROOMIE_CUDA_OK(cudaGetLastError());
+        // One stream, up to 8 slots per GPU.  Two kernels give the same bits: one lane per resident slot (flat in
+        // the admission rate, the shorter chain when most arrivals are admitted) and one lane per modelled GPU
+        // (cheaper while most arrivals are deferred, dearer with every admission).  A long stream starts on the
+        // first kind; every kPlaceWindow arrivals the running kernel looks at the admissions of the window and,
+        // when the other kind suits them better, writes the state back, leaves the number of arrivals done and the
+        // kind that continues in the stream's last gpu_out element and returns.  The launches alternate between
+        // the kinds; one that finds a decision in that element (the stream is done) or a hand-over to the other
+        // kind returns at once, and the last one finishes the stream whatever the rate.
+        PlaceArgs slots = a, fast = a;
+        slots.matrix_mode = 1; slots.pair_cache = 1; slots.gpus_per_warp = 32 / kSlotLanes; slots.chunk = kSlotChunk;
+        slots.my_kind = 1;
+        const uint32_t s_threads = ((a.G * kSlotLanes + 31) / 32) * 32 + 32;   // one more warp that owns no GPU
+        const size_t s_bytes = (size_t)slot_layout(s_threads, a.G).total * sizeof(float);
+        auto s_kern = plain ? place_slots_kernel<true> : place_slots_kernel<false>;
+        if (s_bytes > 48 * 1024)
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(s_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s_bytes));
+        fast.matrix_mode = 1; fast.pair_cache = 1; fast.gpus_per_warp = 32; fast.chunk = kArrChunk;
+        fast.my_kind = 0;
+        const size_t fGR = (size_t)a.G * a.R;
+        const size_t f_bytes = fGR * 5 * 4 + fGR * a.R * 4 + 4 * 2 * fGR * 4 + (kYoungRing * kYoungD * 2 + 2) * 4 +
+                               2 * a.G * 4 + (5 * fast.chunk + 2 * kLead) * sizeof(int32_t);
+        const uint32_t f_threads = 2 * 32 * ((a.G + 31) / 32);
+        auto f_kern = plain ? place_fast_kernel<true> : place_fast_kernel<false>;
+        const bool adaptive = n >= kPlaceAdaptiveFrom && f_bytes <= 160 * 1024;
+        if (adaptive && f_bytes > 48 * 1024)
+            ROOMIE_CUDA_OK(cudaFuncSetAttribute(f_kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)f_bytes));
+        const int launches = adaptive ? kPlaceLaunches : 1;
+        for (int l = 0; l < launches; ++l) {
+            PlaceArgs& k = (l & 1) ? fast : slots;
+            k.mailbox = adaptive ? gpu_out + n - 1 : nullptr;
+            k.first = l == 0; k.may_hand_over = l + 1 < launches;
+            if (l & 1) f_kern<<<1, f_threads, f_bytes, st>>>(k);
+            else s_kern<<<1, s_threads, s_bytes, st>>>(k);
+            note_launch();
+            ROOMIE_CUDA_OK(cudaGetLastError());
+        }
         return ROOMIE_OK;
     }
     const size_t GR = (size_t)a.G * a.R;
@@ -696,7 +789,7 @@ static int place_impl(const float* Pmat, uint32_t P, const roomie_cluster_state*
         a.matrix_mode = 1; a.pair_cache = 1;
         a.gpus_per_warp = 32;
         const uint32_t threads = 2 * 32 * ((a.G + 31) / 32);                 // owner warps + as many fetch warps
-        auto kern = (a.admit_rule == 0 && a.objective == 0) ? place_fast_kernel<true> : place_fast_kernel<false>;
+        auto kern = plain ? place_fast_kernel<true> : place_fast_kernel<false>;
         if (fast_bytes > 48 * 1024)
             ROOMIE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fast_bytes));
         kern<<<num_streams, threads, fast_bytes, st>>>(a);

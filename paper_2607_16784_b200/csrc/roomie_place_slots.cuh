@@ -30,7 +30,7 @@
 constexpr int kSlotLanes = 8;                  // lanes (= resident slots) per modelled GPU
 constexpr int kSlotAhead = 5;                  // arrivals fetched ahead
 constexpr int kSlotStages = 8;                 // ring stages (a power of two > kSlotAhead)
-constexpr uint32_t kSlotChunk = 512;           // arrivals staged in shared memory at a time
+constexpr uint32_t kSlotChunk = 1024;          // arrivals staged in shared memory at a time (= the window between two looks at the admission rate)
 constexpr int kSlotLead = kSlotAhead;          // arrival ids staged before and after a chunk
 constexpr uint32_t kSlotNever = 0xffffffffu;   // expiry tick of a resident that never leaves
 constexpr int32_t kSlotBornLongAgo = -(1 << 30);
@@ -54,6 +54,9 @@ __host__ __device__ inline SlotLayout slot_layout(uint32_t threads, uint32_t G) 
 template <bool kPlain>
 __global__ void __launch_bounds__(1024) place_slots_kernel(PlaceArgs g) {
     select_stream(g);
+    uint32_t k_begin;
+    if (!place_start(g, k_begin)) return;                                 // not this launch's turn
+    __shared__ uint32_t s_placed;
     extern __shared__ __align__(16) float sm[];
     int32_t* smi = reinterpret_cast<int32_t*>(sm);
     const uint32_t G = g.G, R = g.R, P = g.P, n = g.n;
@@ -102,7 +105,7 @@ __global__ void __launch_bounds__(1024) place_slots_kernel(PlaceArgs g) {
     }
     uint32_t cb = __reduce_max_sync(kFull, c);                            // most residents on a GPU of this warp
     const float* my_row = Pm + (size_t)max(id, 0) * P;                    // P[my resident][*]
-    const uint32_t tick0 = *g.tick;
+    const uint32_t tick0 = *g.tick - k_begin;                             // tick of the stream's first arrival
     const uint32_t oRING = L.ring + tid;                                  // + (stage * 2 + dir) * threads
 
     // what arrival a (staged index a_local) will need of this lane's resident, and of the arrivals just before it
@@ -128,7 +131,8 @@ __global__ void __launch_bounds__(1024) place_slots_kernel(PlaceArgs g) {
         cp_async_commit();
     };
 
-    for (uint32_t k0 = 0; k0 < n; k0 += kSlotChunk) {
+    uint32_t k_end = n;                                                   // where this launch stops
+    for (uint32_t k0 = k_begin; k0 < n; k0 += kSlotChunk) {
         const uint32_t kn = min(kSlotChunk, n - k0);
         // stage arrival ids [k0 - lead, k0 + kn + lead) and lifetimes [k0, k0 + kn)
         __syncthreads();
@@ -140,9 +144,9 @@ __global__ void __launch_bounds__(1024) place_slots_kernel(PlaceArgs g) {
         }
         for (uint32_t i = tid; i < kn; i += blockDim.x) smi[L.life + i] = (int32_t)g.arr_life[k0 + i];
         __syncthreads();
-        if (k0 == 0) {                                                    // prime: arrivals 0 .. kAhead-1
+        if (k0 == k_begin) {                                              // prime: the first kAhead arrivals of this launch
             for (uint32_t a = 0; a < (uint32_t)kSlotAhead; ++a) {
-                if (a < n) prefetch(a + kSlotLead, a); else cp_async_commit();
+                if (k_begin + a < n) prefetch(a + kSlotLead, k_begin + a); else cp_async_commit();
             }
             cp_async_wait<0>();
             __syncthreads();
@@ -261,6 +265,13 @@ __global__ void __launch_bounds__(1024) place_slots_kernel(PlaceArgs g) {
             if (g.mean_out) g.mean_out[k0 + i] = sm[L.out + kSlotChunk + i];
             if (g.mu_arr_out) g.mu_arr_out[k0 + i] = sm[L.out + 2 * kSlotChunk + i];
         }
+        // a look at the admission rate: should the other kind of kernel take the rest of the stream?
+        const uint32_t done = k0 + kn;
+        if (g.mailbox && g.may_hand_over && done < n && kn == kPlaceWindow) {
+            uint32_t mine = 0;
+            for (uint32_t i = tid; i < kn; i += blockDim.x) mine += smi[L.out + i] >= 0 ? 1u : 0u;
+            if (kind_for(block_count(mine, &s_placed), kn, g.my_kind) != g.my_kind) { k_end = done; break; }
+        }
     }
     cp_async_wait<0>();
     // ---- write back in arrival order: position t of the list holds slot s ----
@@ -274,5 +285,8 @@ __global__ void __launch_bounds__(1024) place_slots_kernel(PlaceArgs g) {
                 g.expiry[gpu * R + t] = ex == kSlotNever ? 0u : ex;
             }
     }
-    if (tid == 0) *g.tick = tick0 + n;
+    if (tid == 0) {
+        *g.tick = tick0 + k_end;
+        if (k_end < n) g.mailbox[0] = hand_over_word(k_end, 1 - g.my_kind);
+    }
 }
