@@ -426,7 +426,7 @@ def test_placement_rejects_ids_outside_the_matrix(rm, oracle):
     rng = np.random.default_rng(2)
     P = 24
     Pm = (rng.random((P, P)) * 0.2).astype(np.float32)
-    for G, R in ((64, 8), (6, 12)):                                   # fast kernel, generic kernel
+    for G, R in ((64, 8), (6, 12)):                                   # slot kernel, generic kernel (one lane per GPU: the long-stream test below)
         n = 200
         aid = rng.integers(0, P, n).astype(np.int32)
         life = rng.integers(1, 40, n).astype(np.uint32)
@@ -456,6 +456,50 @@ def test_placement_rejects_ids_outside_the_matrix(rm, oracle):
         st = rm.ClusterState(G, R, ids0, [0] * (G * R), cnt0, 0)
         gpu = rm.place(Pm, st, aid, life, 0.5)[0].cpu().numpy()
         assert (gpu == -2).all() and np.array_equal(st.ids.cpu().numpy(), ids0) and int(st.tick.item()) == 0
+
+
+def test_placement_long_stream_changes_kernels(rm, oracle):
+    """A single stream of 4 096 arrivals or more changes between the two single-stream kernels with the admission rate
+    (looked at every 1 024 arrivals), the cluster state going through the caller's arrays at every change.  This
+    stream forces the changes: every arrival is admitted while slots are free (lambda is huge), the first 2 000 stay
+    for 6 000 ticks, so the cluster (16 GPUs x 4 slots) is full from arrival 64 on and nothing is admitted until tick
+    6 000 (one lane per GPU takes over), then a slot frees with every tick and every arrival is admitted again for a
+    while (one lane per slot takes over), with residents leaving in every phase.  Decisions, means and the final state
+    must equal the oracle's; and with ids outside the matrix sprinkled over all phases, those arrivals are refused and
+    the rest is as if they had only taken their tick."""
+    rng = np.random.default_rng(5)
+    P, n, G, R = 48, 12000, 16, 4
+    Pm = (rng.random((P, P)) * 0.3).astype(np.float32)
+    aid = rng.integers(0, P, n).astype(np.int32)
+    life = np.where(np.arange(n) < 2000, 6000, rng.integers(1, 50, n)).astype(np.uint32)
+    empty = ([-1] * (G * R), [0] * (G * R), [0] * G)
+    st = rm.ClusterState(G, R, *empty, 0)
+    gpu, mean, _ = rm.place(Pm, st, aid, life, 1e9)
+    gpu = gpu.cpu().numpy()
+    want = oracle.place(Pm, G, R, *empty, 0, aid, life, 1e9)
+    assert np.array_equal(gpu, want.gpu)
+    assert np.array_equal(mean.cpu().numpy().view(np.uint32), want.mean.view(np.uint32))
+    assert np.array_equal(st.ids.cpu().numpy(), want.ids) and np.array_equal(to_np_u32(st.expiry), want.expiry)
+    assert np.array_equal(to_np_u32(st.count), want.count) and int(st.tick.item()) == n
+    # the phases are there: all admitted, none, all again
+    adm = (gpu >= 0).reshape(-1, 1000).mean(axis=1)
+    assert adm[0] < 0.1 and adm[1:5].max() == 0.0 and adm[6] == 1.0, adm
+    bad_at = [3, 1500, 2047, 2048, 4096, 6500, 11999]
+    bad = aid.copy()
+    bad[bad_at] = [P, -1, P + 5, 1 << 30, -7, P, P]
+    st = rm.ClusterState(G, R, *empty, 0)
+    gpu = rm.place(Pm, st, bad, life, 1e9)[0].cpu().numpy()
+    ids, exp, cnt = empty
+    want_gpu = np.full(n, -2, np.int32)
+    start = 0
+    for stop in bad_at + [n]:                                         # the stretches between the refused arrivals
+        if stop > start:
+            w = oracle.place(Pm, G, R, ids, exp, cnt, start, aid[start:stop], life[start:stop], 1e9)
+            want_gpu[start:stop] = w.gpu
+            ids, exp, cnt = w.ids, w.expiry, w.count
+        start = stop + 1                                              # a refused arrival still takes its tick
+    assert np.array_equal(gpu, want_gpu)
+    assert int(st.tick.item()) == n
 
 
 # ----------------------------------------------------------------------------- placement variants, batches
