@@ -114,16 +114,13 @@ typedef struct roomie_library {
     uint32_t *offsets;            /* device [P+1]                                                */
     void *records;                /* device [K] x 16 bytes, 16-byte aligned                      */
     uint64_t *T;                  /* device [P] isolated inference time = sum of kernel ticks     */
-    float *share_table;           /* device [roomie_share_table_floats(spec)] occupancy shares   */
     uint32_t *status;             /* device [1] sticky ROOMIE_FLAG_* bits; zero it before build   */
     roomie_gpu_spec spec;
 } roomie_library;
 
-/* Number of floats of roomie_library.share_table for a spec: 2W + 1, W = threads_per_sm/32.
- * Entry s holds 1/s (entry 0 is 0): the occupancy share o_i/(o_i+o_j) of Algorithm 1 line 13
- * equals warps_i * table[warps_i + warps_j] (W cancels); a charged delay is evaluated as
- * (ticks * table[...]) * warps_i in float32. */
-size_t roomie_share_table_floats(const roomie_gpu_spec *spec /* host */);
+/* The occupancy share o_i/(o_i+o_j) of Algorithm 1 line 13 is evaluated from the resident warps of
+ * the two kernels (W cancels): a charged delay is (ticks * (1/(warps_i + warps_j))) * warps_i in
+ * float32, the reciprocal to one unit in the last place. */
 
 /* Builds the library from a kernel table plus isolated durations and inter-kernel gaps
  * (microseconds, float32, device arrays [K]).  Times become integer ticks of 1 ns:

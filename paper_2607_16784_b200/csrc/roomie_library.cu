@@ -178,13 +178,6 @@ __global__ void __launch_bounds__(kBuildThreads) library_build_kernel(BuildArgs 
     if (threadIdx.x == 0) a.T[m] = sum_d;
 }
 
-// Reciprocals 1/s for every possible sum of two warp counts: the occupancy share of
-// Algorithm 1 line 13 is o_i/(o_i+o_j) = warps_i * (1 / (warps_i + warps_j)).
-__global__ void share_table_kernel(float* tab, uint32_t n) {
-    const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
-    if (s < n) tab[s] = s ? __frcp_rn((float)s) : 0.0f;
-}
-
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Which occupancy kernel a call gets (pointers are only looked at, never dereferenced):
@@ -248,17 +241,12 @@ extern "C" int roomie_occupancy_variant(const roomie_kernel_table* table, const 
     return occupancy_variant_of(table, out);
 }
 
-extern "C" size_t roomie_share_table_floats(const roomie_gpu_spec* spec) {
-    if (validate_spec(spec) != ROOMIE_OK) return 0;
-    return 2 * (size_t)(spec->threads_per_sm / 32u) + 1u;
-}
-
 extern "C" int roomie_library_build(const roomie_library* lib, const roomie_kernel_table* table,
                                     const float* dur_us, const float* gap_us, void* stream) {
     if (!lib || !table || !dur_us || !gap_us) return ROOMIE_ERR_INVALID_ARG;
     const int vs = validate_spec(&lib->spec);
     if (vs != ROOMIE_OK) return vs;
-    if (!lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->share_table || !lib->status)
+    if (!lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->status)
         return ROOMIE_ERR_INVALID_ARG;
     if (lib->num_profiles == 0 || table->n != lib->num_kernels || lib->offsets_host[0] != 0 ||
         lib->offsets_host[lib->num_profiles] != lib->num_kernels || !aligned16(lib->records))
@@ -278,10 +266,6 @@ extern "C" int roomie_library_build(const roomie_library* lib, const roomie_kern
     a.T = reinterpret_cast<unsigned long long*>(lib->T);
     a.status = lib->status; a.spec = lib->spec;
     library_build_kernel<<<lib->num_profiles, kBuildThreads, 0, st>>>(a);
-    note_launch();
-    ROOMIE_CUDA_OK(cudaGetLastError());
-    const uint32_t n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u;
-    share_table_kernel<<<(n_inv + 255) / 256, 256, 0, st>>>(lib->share_table, n_inv);
     note_launch();
     ROOMIE_CUDA_OK(cudaGetLastError());
     return ROOMIE_OK;

@@ -205,8 +205,6 @@ struct TileArgs {
     const uint32_t* tile_counter;
     uint32_t tile_capacity;
     TilePartial* partials;
-    const float* inv_table;      // [2W + 1] 1/s (LOCKSTEP tiles only)
-    uint32_t n_inv;              // 2W + 1
     PhiCap cap;
     uint32_t* status;            // library status word (sticky flags)
 };
@@ -424,11 +422,11 @@ __global__ void __launch_bounds__(kTileThreads) lockstep_tiles_kernel(TileArgs g
         for (uint32_t i = threadIdx.x; i < d.cntA; i += kTileThreads) {
             const uint4 ra = __ldg(&g.records[d.recA + i]), rb = __ldg(&g.records[d.recB + i]);
             if (phi_exceeds(g.cap.lo - ra.z, g.cap.hi - ra.w, rb.z, rb.w)) {
-                const uint32_t wa = ra.z >> kWarpShift, wb = rb.z >> kWarpShift;
-                const float inv = __ldg(&g.inv_table[wa + wb]);
+                const float wa = small_int_to_float(ra.z >> kWarpShift), wb = small_int_to_float(rb.z >> kWarpShift);
+                const float inv = fast_rcp(wa + wb);              // an interfering pair has resident warps on both sides
                 const uint32_t da = ra.y - ra.x, db = rb.y - rb.x;
-                di = fmaf((float)da * inv, small_int_to_float(wa), di);
-                dj = fmaf((float)db * inv, small_int_to_float(wb), dj);
+                di = fmaf((float)da * inv, wa, di);
+                dj = fmaf((float)db * inv, wb, dj);
                 V += (unsigned long long)da + db;
             }
         }
@@ -761,7 +759,7 @@ static int run_lockstep_full(const roomie_library* lib, const roomie_opts* o, co
 static bool wants_lockstep_full(const roomie_opts* o) { return o->walk_mode == ROOMIE_WALK_LOCKSTEP && o->n_align == 0; }
 
 static int check_lib(const roomie_library* lib, const roomie_opts* o) {
-    if (!lib || !o || !lib->offsets_host || !lib->offsets || !lib->records || !lib->T || !lib->share_table ||
+    if (!lib || !o || !lib->offsets_host || !lib->offsets || !lib->records || !lib->T ||
         !lib->status || lib->num_profiles == 0)
         return ROOMIE_ERR_INVALID_ARG;
     // 16-byte loads and bulk copies of the records: a misaligned table would fault on the device
@@ -862,8 +860,7 @@ static int run_batch(const roomie_library* lib, const roomie_opts* o, const Pair
 
     TileArgs ta;
     ta.records = lv.records; ta.tiles = tiles; ta.tile_counter = counter; ta.tile_capacity = (uint32_t)need.tiles; ta.partials = partials;
-    ta.inv_table = lib->share_table;
-    ta.n_inv = 2u * (lib->spec.threads_per_sm / 32u) + 1u; ta.cap = lv.cap; ta.status = lib->status;
+    ta.cap = lv.cap; ta.status = lib->status;
     profile_mark(st, true);
     if (pa.lockstep) {
         uint64_t grid = (uint64_t)sm_count() * 8;

@@ -15,7 +15,7 @@ TIMELINE, LOCKSTEP = 0, 1
 DETAILED_EQUAL, DETAILED_PRIORITY, DETAILED_FCFS = 2, 3, 4
 
 EXPORTS = [
-    "roomie_occupancy", "roomie_occupancy_variant", "roomie_share_table_floats", "roomie_library_build",
+    "roomie_occupancy", "roomie_occupancy_variant", "roomie_library_build",
     "roomie_pair_workspace_bytes", "roomie_pair_matrix", "roomie_pair_interference",
     "roomie_pair_interference_workspace_bytes", "roomie_selftest_bounded_wait",
     "roomie_pair_interference_static",
@@ -42,7 +42,6 @@ def _load():
     dll.roomie_strerror.restype = C.c_char_p
     dll.roomie_last_cuda_error.restype = C.c_char_p
     dll.roomie_launch_count.restype = C.c_uint64
-    dll.roomie_share_table_floats.restype = C.c_size_t
     dll.roomie_pair_workspace_bytes.restype = C.c_size_t
     dll.roomie_pair_workspace_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64]
     dll.roomie_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
@@ -100,7 +99,7 @@ class _OccOut(C.Structure):
 class _Library(C.Structure):
     _fields_ = [("num_profiles", C.c_uint32), ("num_kernels", C.c_uint32),
                 ("offsets_host", C.c_void_p), ("offsets", C.c_void_p), ("records", C.c_void_p),
-                ("T", C.c_void_p), ("share_table", C.c_void_p), ("status", C.c_void_p), ("spec", _Spec)]
+                ("T", C.c_void_p), ("status", C.c_void_p), ("spec", _Spec)]
 
 
 class _Opts(C.Structure):
@@ -198,12 +197,9 @@ class Library:
         self.records = torch.empty((K, 4), dtype=torch.int32, device=device)
         self.T = torch.empty(P, dtype=torch.int64, device=device)
         cs = _cspec(spec)
-        self.share_table = torch.empty(int(_dll.roomie_share_table_floats(C.byref(cs))),
-                                       dtype=torch.float32, device=device)
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
         self.c = _Library(P, K, self.offsets_host.ctypes.data, self.offsets.data_ptr(),
-                          self.records.data_ptr(), self.T.data_ptr(), self.share_table.data_ptr(),
-                          self.status.data_ptr(), cs)
+                          self.records.data_ptr(), self.T.data_ptr(), self.status.data_ptr(), cs)
 
     def status_flags(self) -> int:
         """Synchronises and returns the sticky ROOMIE_FLAG_* bits."""

@@ -38,12 +38,6 @@ def test_host_side_argument_checks():
     assert dll.roomie_library_build(None, None, None, None, None) == -1
     assert dll.roomie_place(None, 0, None, None, None, 0, None, None, None, None, None) == -1
 
-    class Spec(ctypes.Structure):
-        _fields_ = [(n, ctypes.c_uint32) for n in "abcde"]
-    dll.roomie_share_table_floats.restype = ctypes.c_size_t
-    assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 65536, 164 * 1024, 2048, 32))) == 2 * 64 + 1
-    assert dll.roomie_share_table_floats(ctypes.byref(Spec(108, 1 << 18, 164 * 1024, 2048, 32))) == 0   # RANGE
-
 
 def test_workspace_size_queries_are_host_only():
     """The two size queries read only the host copy of the profile offsets: they answer without a GPU, agree with
@@ -61,7 +55,7 @@ def test_workspace_size_queries_are_host_only():
     fake = 0x10000                                           # never dereferenced by the size queries
 
     def library(records_ptr):
-        return rm._Library(3, 9000, offsets.ctypes.data, fake, records_ptr, fake, fake, fake,
+        return rm._Library(3, 9000, offsets.ctypes.data, fake, records_ptr, fake, fake,
                            rm._Spec(108, 65536, 164 * 1024, 2048, 32))
 
     def opts(mode, n_align):
