@@ -335,14 +335,25 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
     __shared__ unsigned long long s_v[kTileThreads / 32];
     __shared__ uint32_t s_t[kTileThreads / 32];
 
+    __shared__ TileDesc s_desc[2];                         // this tile's descriptor and the next one's, fetched ahead
     if (threadIdx.x == 0) mbar_init(&s_bar, 1);
-    __syncthreads();
     const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
+    if (threadIdx.x == 0 && blockIdx.x < n_tiles) s_desc[0] = g.tiles[blockIdx.x];
+    __syncthreads();
     const PhiCap cap = g.cap;
-    uint32_t parity = 0;
+    uint32_t parity = 0, buf = 0;
 
-    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        const TileDesc d = g.tiles[t];
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, buf ^= 1u) {
+        const TileDesc d = s_desc[buf];
+        if (threadIdx.x == 32) {                           // the next descriptor arrives while this tile is walked
+            if (t + gridDim.x < n_tiles) {
+                const uint32_t dst = smem_addr(&s_desc[buf ^ 1u]);
+                const TileDesc* src = &g.tiles[t + gridDim.x];
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst + 16u), "l"(reinterpret_cast<const char*>(src) + 16) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
         const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
         const uint32_t b_off = (loadA + kChunk - 1) & ~(uint32_t)(kChunk - 1);
         if (threadIdx.x == 0) mbar_arrive_expect(&s_bar, (loadA + loadB) * (uint32_t)sizeof(uint4));
@@ -386,6 +397,7 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
                 for (int s = 0; s < kItems; ++s) ROOMIE_WALK_STEP((uint32_t)s < steps)
             }
         }
+        if (threadIdx.x == 32) asm volatile("cp.async.wait_group 0;" ::: "memory");   // before the barrier inside the reduction
         block_reduce_store<kWithV>(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
     }
 }
