@@ -338,15 +338,30 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
     __shared__ TileDesc s_desc[2];                         // this tile's descriptor and the next one's, fetched ahead
     if (threadIdx.x == 0) mbar_init(&s_bar, 1);
     const uint32_t n_tiles = min(*g.tile_counter, g.tile_capacity);
-    if (threadIdx.x == 0 && blockIdx.x < n_tiles) s_desc[0] = g.tiles[blockIdx.x];
+    if (blockIdx.x >= n_tiles) return;
+    if (threadIdx.x == 0) s_desc[0] = g.tiles[blockIdx.x];
     __syncthreads();
     const PhiCap cap = g.cap;
     uint32_t parity = 0, buf = 0;
+    // The records of a tile are on their way before the CTA turns to it: those of the first tile from here, those
+    // of every later one from the end of the walk before it (the tile's sums are still being added up then).
+    auto expect_tile = [&](const TileDesc& dn) {           // one thread: the bytes the barrier will see
+        const uint32_t la = dn.cntA + (dn.flags & 1u), lb = dn.cntB + ((dn.flags >> 1) & 1u);
+        mbar_arrive_expect(&s_bar, (la + lb) * (uint32_t)sizeof(uint4));
+    };
+    auto stage_tile = [&](const TileDesc& dn) {            // every thread: its share of the bulk copies
+        const uint32_t la = dn.cntA + (dn.flags & 1u), lb = dn.cntB + ((dn.flags >> 1) & 1u);
+        stage_tile_async(g.records, dn, la, lb, (la + kChunk - 1) & ~(uint32_t)(kChunk - 1), s_rec, &s_bar);
+    };
+    if (threadIdx.x == 32) expect_tile(s_desc[0]);
+    __syncthreads();
+    stage_tile(s_desc[0]);
 
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, buf ^= 1u) {
         const TileDesc d = s_desc[buf];
+        const bool more = t + gridDim.x < n_tiles;
         if (threadIdx.x == 32) {                           // the next descriptor arrives while this tile is walked
-            if (t + gridDim.x < n_tiles) {
+            if (more) {
                 const uint32_t dst = smem_addr(&s_desc[buf ^ 1u]);
                 const TileDesc* src = &g.tiles[t + gridDim.x];
                 asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
@@ -354,11 +369,8 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        const uint32_t loadA = d.cntA + (d.flags & 1u), loadB = d.cntB + ((d.flags >> 1) & 1u);
+        const uint32_t loadA = d.cntA + (d.flags & 1u);
         const uint32_t b_off = (loadA + kChunk - 1) & ~(uint32_t)(kChunk - 1);
-        if (threadIdx.x == 0) mbar_arrive_expect(&s_bar, (loadA + loadB) * (uint32_t)sizeof(uint4));
-        __syncthreads();                                   // previous tile fully consumed
-        stage_tile_async(g.records, d, loadA, loadB, b_off, s_rec, &s_bar);
         const bool arrived = mbar_wait_bounded(&s_bar, parity);
         parity ^= 1u;
         if (!__syncthreads_and(arrived)) {
@@ -397,7 +409,12 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
                 for (int s = 0; s < kItems; ++s) ROOMIE_WALK_STEP((uint32_t)s < steps)
             }
         }
-        if (threadIdx.x == 32) asm volatile("cp.async.wait_group 0;" ::: "memory");   // before the barrier inside the reduction
+        if (threadIdx.x == 32) {                           // (its own copy of the next descriptor has landed)
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            if (more) expect_tile(s_desc[buf ^ 1u]);
+        }
+        __syncthreads();                                   // this tile's records are consumed, the next descriptor is in place
+        if (more) stage_tile(s_desc[buf ^ 1u]);
         block_reduce_store<kWithV>(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
     }
 }
