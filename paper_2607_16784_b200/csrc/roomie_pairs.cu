@@ -371,22 +371,17 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
         }
         const uint32_t loadA = d.cntA + (d.flags & 1u);
         const uint32_t b_off = (loadA + kChunk - 1) & ~(uint32_t)(kChunk - 1);
+        // a thread whose wait has succeeded sees the tile's records; whether every thread's has is settled at the
+        // barrier after the walk
         const bool arrived = mbar_wait_bounded(&s_bar, parity);
         parity ^= 1u;
-        if (!__syncthreads_and(arrived)) {
-            // a copy did not arrive within the bound: report it, give the copies in flight one more
-            // bounded wait so that none lands after the CTA has gone, and stop
-            if (threadIdx.x == 0) atomicOr(g.status, ROOMIE_FLAG_WAIT_TIMEOUT);
-            if (!arrived) mbar_wait_bounded(&s_bar, parity ^ 1u);
-            return;
-        }
         const uint32_t len = d.cntA + d.cntB;
         const uint32_t diag = threadIdx.x * kItems;
         const uint32_t delta = d.baseA - d.baseB;          // B tick + delta = the same instant in A's ticks
         float di = 0.0f, dj = 0.0f;
         unsigned long long V = 0;
         uint32_t ties = 0;
-        if (diag < len) {
+        if (arrived && diag < len) {
             // this thread's start point on the tile's merge path (A first on equal end times):
             // B record y sits at unified index b_off + y
             uint32_t lo = diag > d.cntB ? diag - d.cntB : 0u, hi = diag < d.cntA ? diag : d.cntA;
@@ -411,9 +406,16 @@ __global__ void __launch_bounds__(kTileThreads, kTileCtasPerSm) timeline_tiles_k
         }
         if (threadIdx.x == 32) {                           // (its own copy of the next descriptor has landed)
             asm volatile("cp.async.wait_group 0;" ::: "memory");
-            if (more) expect_tile(s_desc[buf ^ 1u]);
+            if (more && arrived) expect_tile(s_desc[buf ^ 1u]);
         }
-        __syncthreads();                                   // this tile's records are consumed, the next descriptor is in place
+        // this tile's records are consumed, the next descriptor is in place
+        if (!__syncthreads_and(arrived)) {
+            // a copy did not arrive within the bound: report it, give the copies in flight one more
+            // bounded wait so that none lands after the CTA has gone, and stop (nothing of the next tile is in flight)
+            if (threadIdx.x == 0) atomicOr(g.status, ROOMIE_FLAG_WAIT_TIMEOUT);
+            if (!arrived) mbar_wait_bounded(&s_bar, parity ^ 1u);
+            return;
+        }
         if (more) stage_tile(s_desc[buf ^ 1u]);
         block_reduce_store<kWithV>(di, dj, V, ties, &g.partials[t], s_f, s_v, s_t, kTileThreads / 32);
     }
