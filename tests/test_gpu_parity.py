@@ -484,6 +484,17 @@ def test_placement_long_stream_changes_kernels(rm, oracle):
     # the phases are there: all admitted, none, all again
     adm = (gpu >= 0).reshape(-1, 1000).mean(axis=1)
     assert adm[0] < 0.1 and adm[1:5].max() == 0.0 and adm[6] == 1.0, adm
+    # admissions that swing with every window of 1 024 arrivals (lifetimes of 200 ticks: a third admitted; of 30: all),
+    # more swings than there are launches to hand over to: the last launch finishes the stream whatever the rate
+    life2 = np.where((np.arange(n) // 1024) % 2 == 0, 200, 30).astype(np.uint32)
+    st = rm.ClusterState(G, R, *empty, 0)
+    gpu2, mean2, _ = rm.place(Pm, st, aid, life2, 1e9)
+    want2 = oracle.place(Pm, G, R, *empty, 0, aid, life2, 1e9)
+    assert np.array_equal(gpu2.cpu().numpy(), want2.gpu)
+    assert np.array_equal(mean2.cpu().numpy().view(np.uint32), want2.mean.view(np.uint32))
+    assert np.array_equal(st.ids.cpu().numpy(), want2.ids) and np.array_equal(to_np_u32(st.expiry), want2.expiry)
+    adm2 = (want2.gpu >= 0).reshape(-1)[:11 * 1024].reshape(11, 1024).mean(axis=1)
+    assert adm2[2::2].max() < 0.45 and adm2[1::2].min() > 0.55, adm2
     bad_at = [3, 1500, 2047, 2048, 4096, 6500, 11999]
     bad = aid.copy()
     bad[bad_at] = [P, -1, P + 5, 1 << 30, -7, P, P]
